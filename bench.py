@@ -1,0 +1,396 @@
+#!/usr/bin/env python
+"""Benchmark of the tool-tracking hot path: frames/s over K concurrent streams, per-frame latency
+distribution at a 16.7 ms frame period, and achieved fraction of the B200 roofline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--streams S]
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference     # the CPU oracle timed on the host cores
+
+One "step" is one tick: the newest frame of every stream goes through the whole path
+(preprocess, encoder, ConvLSTM step, postprocess, optional overlay).  `value` is whole-job
+frames/s with the frames already resident in HBM, timed on the device with CUDA events on the
+launching stream; `e2e` is the same metric through tt_submit_frames/tt_sync with pinned host
+frames (host->device copies and the device->host result read inside the timed region).
+Streams are independent, so with N GPUs every rank runs its own K streams (weak scaling, no
+data-path collective); the reported time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "frames/s over K streams"
+UNIT = "frames/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+FRAME_PERIOD_NS = 16_666_667
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"]))}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+def describe(wl, K):
+    return (f"{wl.name}: K={K} concurrent streams, {wl.src_w}x{wl.src_h} uint8 RGB -> {wl.net_w}x{wl.net_h}, "
+            f"encoder 3->{'->'.join(str(c) for c in wl.enc_cout)} (strides {list(wl.enc_stride)}), "
+            f"ConvLSTM hidden {wl.hidden} on {wl.map_hw()[1]}x{wl.map_hw()[0]}, {wl.n_tools} tools, {wl.precision}"
+            + (", overlay on" if wl.overlay else ""))
+
+
+# ------------------------------------------------------------------------------ work model
+def stage_work(wl, K):
+    """Algorithmic bytes / flops of each stage for one tick of K stream-frames."""
+    hm, wm = wl.map_hw()
+    plane = hm * wm
+    out = {}
+    out["preprocess"] = {"bound": "hbm", "bytes": K * (3 * wl.src_w * wl.src_h + 12 * wl.net_w * wl.net_h)}
+    h, w, cin = wl.net_h, wl.net_w, 3
+    act_bytes = 2 if wl.precision == "bf16" else 4
+    for l, (co, s) in enumerate(zip(wl.enc_cout, wl.enc_stride)):
+        ho, wo = (h + 2 - 3) // s + 1, (w + 2 - 3) // s + 1
+        flops = 2.0 * K * ho * wo * co * 9 * cin
+        in_bytes = K * h * w * cin * (4 if l == 0 else act_bytes)
+        out_bytes = K * ho * wo * co * act_bytes
+        if l == 0 or wl.precision != "bf16":
+            out[f"enc{l}"] = {"bound": "hbm" if l == 0 else "alu", "bytes": in_bytes + out_bytes, "flops": flops}
+        else:
+            out[f"enc{l}"] = {"bound": "tensor", "flops": flops, "bytes": in_bytes + out_bytes}
+        h, w, cin = ho, wo, co
+    ch = wl.hidden
+    out["convlstm"] = {"bound": "tensor" if wl.precision == "bf16" else "alu",
+                       "flops": 2.0 * K * plane * 4 * ch * 9 * (cin + ch),
+                       "bytes": K * plane * (cin * act_bytes + ch * act_bytes + 8 * ch + 4 * ch + 2 * ch)}
+    out["postprocess"] = {"bound": "hbm", "bytes": K * plane * (4 * ch + wl.n_tools * 9 + 1)}
+    if wl.overlay:
+        out["overlay"] = {"bound": "hbm", "bytes": K * (7 * wl.src_w * wl.src_h + plane)}
+    return out
+
+
+# ---------------------------------------------------------------------------- clock sampling
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        cmd = ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100"]
+        if uuid:
+            cmd += ["-i", uuid]
+        try:
+            self.proc = subprocess.Popen(cmd, stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        rows = [r.strip().split(", ") for r in open(self.tmp.name).read().splitlines() if r.strip()]
+        os.unlink(self.tmp.name)
+        sm, reasons, smax = [], set(), None
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1])); smax = float(r[2])
+            except ValueError:
+                continue
+            for name, v in zip(names, r[5:9]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            sm.sort()
+            out.update({"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": smax, "reasons": sorted(reasons), "samples": len(sm)})
+        return out
+
+
+# ------------------------------------------------------------------------------ CPU oracle
+def time_oracle(wl, budget_s=12.0, max_frames=8):
+    """The oracle as it stands, on a bounded sample: whole stream-frames of this workload."""
+    import oracle
+    import tt_synth
+    w = tt_synth.make_weights(wl)
+    pipe = oracle.OraclePipeline(wl, w)
+    n, t_total = 0, 0.0
+    while n < max_frames and (n == 0 or t_total < budget_s):
+        fr = tt_synth.make_frame(wl.frame_kind, wl.stream_seed(0), n, wl.src_w, wl.src_h)
+        t0 = time.perf_counter()
+        pipe.step(fr)
+        t_total += time.perf_counter() - t0
+        n += 1
+    return {"value": n / t_total, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{n} stream-frames of {wl.name} (one stream, consecutive frames) in {t_total:.1f} s; "
+                      "per-frame cost is independent of K, so K streams cost K times as much"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    import tt_synth
+    wl = tt_synth.workload(args.workload)
+    K = args.streams or wl.streams
+    w = tt_synth.make_weights(wl)
+    pipe = oracle.OraclePipeline(wl, w)
+    frames = [tt_synth.make_frame(wl.frame_kind, wl.stream_seed(0), t, wl.src_w, wl.src_h) for t in range(4)]
+    for i in range(args.warmup):
+        t0 = time.perf_counter()
+        pipe.step(frames[i % 4])
+        if (time.perf_counter() - t0) * (args.steps + args.warmup - i) > 240 and i >= 0:
+            break
+    times, budget = [], 240.0
+    for i in range(args.steps):
+        t0 = time.perf_counter()
+        pipe.step(frames[i % 4])
+        times.append(time.perf_counter() - t0)
+        if sum(times) > budget:
+            break
+    total = sum(times)
+    value = len(times) / total
+    sample = (f"each step = 1 stream-frame of {wl.name} through the CPU oracle ({oracle.num_threads()} host threads); "
+              f"{len(times)} of {args.steps} requested steps fitted the time budget")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 0, "steps": len(times),
+            "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": describe(wl, K), "note": "one stream-frame per step; oracle cost scales linearly in K"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+# -------------------------------------------------------------------------------- GPU arm
+def run_ours(args):
+    import ctypes as C
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import tt_synth
+    from paper_2402_04466_b200 import binding
+    from paper_2402_04466_b200.stats import latency_summary, trim_warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    wl = tt_synth.workload(args.workload)
+    K = args.streams or wl.streams
+    if args.overlay is not None:
+        wl = wl.with_(overlay=bool(args.overlay))
+    weights = tt_synth.make_weights(wl)
+    stream = torch.cuda.Stream()
+    cfg = binding.make_config(wl, max_streams=K, device=local_rank, cuda_stream=stream.cuda_stream)
+    ctx = binding.Context(cfg, weights)
+    states = [ctx.state_create() for _ in range(K)]
+
+    # ring of distinct frames per stream (seeded; stream s of rank r uses seed index r*K + s)
+    R = args.ring
+    host_ring = [[torch.from_numpy(tt_synth.make_frame(wl.frame_kind, wl.stream_seed(rank * K + s), t, wl.src_w, wl.src_h)).pin_memory()
+                  for t in range(R)] for s in range(K)]
+    dev_ring = [[f.to(dev) for f in host_ring[s]] for s in range(K)]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    frame_bytes = wl.src_h * wl.src_pitch
+
+    def tick(i, ring):
+        ctx.submit_frames([ring[s][i % R] for s in range(K)], states, frame_index=i)
+        return ctx.sync()
+
+    def flush_l2(i):
+        with torch.cuda.stream(stream):
+            flush.fill_(i & 0xFF)
+
+    ctx.set_profiling(True)
+    for i in range(args.warmup):
+        flush_l2(i)
+        tick(i, dev_ring)
+
+    uuid = None
+    try:
+        uuid = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(uuid) if rank == 0 else None
+    launches0, _ = ctx.get_counters()
+
+    # ---- timed region 1: device-resident frames, device time per tick from CUDA events
+    barrier()
+    step_ms, stage_sum = [], {}
+    for i in range(args.steps):
+        flush_l2(i)
+        res = tick(i, dev_ring)
+        step_ms.append(res[0]["gpu_ms"])
+        for k, v in ctx.get_stage_times().items():
+            stage_sum[k] = stage_sum.get(k, 0.0) + v
+    barrier()
+    launches1, _ = ctx.get_counters()
+    total_ms = float(sum(step_ms))
+
+    # ---- timed region 2: end to end through the public calls with pinned host frames
+    barrier()
+    e2e_s = 0.0
+    for i in range(args.steps):
+        flush_l2(i)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        tick(i, host_ring)
+        e2e_s += time.perf_counter() - t0
+    barrier()
+    clocks = sampler.stop() if sampler else None
+
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_s = float(t[0]), float(t[1])
+
+    # ---- paced latency run (rank 0 of a single-GPU job): frames arrive every 16.7 ms per stream
+    latency = None
+    if world == 1 and args.paced_frames > 0:
+        ctx.set_profiling(False)
+        for s in states:
+            ctx.state_reset(s)
+        try:
+            os.sched_setaffinity(0, {sorted(os.sched_getaffinity(0))[-1]})
+        except Exception:
+            pass
+        fr = (binding.tt_frame * K)()
+        sts = (C.c_void_p * K)(*[s.value for s in states])
+        res = (binding.tt_result * binding.TT_MAX_STREAMS)()
+        lat_ms, gpu_ms, misses = [], [], 0
+        t_start = time.perf_counter_ns() + 2_000_000
+        for i in range(args.paced_frames):
+            arrival = t_start + i * FRAME_PERIOD_NS
+            while time.perf_counter_ns() < arrival:
+                pass
+            for s in range(K):
+                fr[s].data = host_ring[s][i % R].data_ptr()
+                fr[s].on_device = 0
+                fr[s].frame_index = i
+                fr[s].arrival_ns = arrival
+            st = ctx.submit_raw(K, fr, sts)
+            st = st or ctx.sync_raw(res)
+            done = time.perf_counter_ns()
+            if st != 0:
+                raise RuntimeError(f"paced run failed: {ctx.last_error()}")
+            lat_ms.append((done - arrival) / 1e6)
+            gpu_ms.append(res[0].gpu_ms)
+            misses += int(done - arrival > FRAME_PERIOD_NS)
+        lat = trim_warmup(lat_ms)
+        latency = latency_summary(lat)
+        latency.update({"streams": K, "frames_per_stream": args.paced_frames, "frame_period_ms": FRAME_PERIOD_NS / 1e6,
+                        "deadline_misses": misses, "gpu_ms_mean": float(np.mean(trim_warmup(gpu_ms))),
+                        "definition": "scheduled arrival of the K frames -> tt_sync returned (pinned host frames, H2D inside)"})
+
+    if rank != 0:
+        ctx.destroy()
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    peaks, peak_kind = load_peaks()
+    work = stage_work(wl, K)
+    stages = {}
+    for name, wk in work.items():
+        if name not in stage_sum:
+            continue
+        ms = stage_sum[name] / args.steps
+        ent = {"ms": ms, "bound": wk["bound"]}
+        if wk["bound"] == "hbm":
+            ent.update({"achieved": wk["bytes"] / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"})
+        elif wk["bound"] == "tensor":
+            ent.update({"achieved": wk["flops"] / (ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"})
+        else:
+            ent.update({"achieved": wk["flops"] / (ms * 1e-3) / 1e12, "peak": None, "unit": "TFLOP/s"})
+        ent["frac"] = ent["achieved"] / ent["peak"] if ent.get("peak") else None
+        stages[name] = ent
+    dom = max(stages, key=lambda n: stages[n]["ms"])
+    d = stages[dom]
+    roofline = {"kernel": dom, "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"], "unit": d["unit"],
+                "frac": d["frac"], "traffic": None, "peak_source": f"of {peak_kind} (burst figure)",
+                "launch_ms": d["ms"]}
+
+    cpu_baseline = time_oracle(wl.with_(overlay=False)) if (world == 1 and not args.no_cpu_baseline) else None
+    n_frames = world * K * args.steps
+    line = {
+        "metric": METRIC, "value": n_frames / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if wl.precision == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": describe(wl, K), "streams_per_gpu": K, "frame_ring": R,
+                   "l2": "flushed between timed steps (256 MiB device write outside the timed events)",
+                   "timing": "CUDA events on the launching stream around every tick, summed over the timed steps"},
+        "e2e": {"value": n_frames / e2e_s, "unit": UNIT, "h2d_bytes_per_step": K * frame_bytes,
+                "d2h_bytes_per_step": K * C.sizeof(binding.tt_result) + 4,
+                "timing": "host clock around tt_submit_frames + tt_sync, pinned host frames"},
+        "gpu_launches": launches1 - launches0,
+        "roofline": roofline, "stages": stages, "clocks": clocks,
+    }
+    if latency is not None:
+        line["latency"] = latency
+    if cpu_baseline is not None:
+        line["cpu_baseline"] = cpu_baseline
+    print(json.dumps(line))
+    ctx.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", help="cfg0..cfg4 (optionally with -gain)")
+    ap.add_argument("--streams", type=int, default=0, help="streams per GPU (default: the workload's)")
+    ap.add_argument("--overlay", type=int, default=None)
+    ap.add_argument("--ring", type=int, default=8, help="distinct frames per stream, reused cyclically")
+    ap.add_argument("--paced-frames", type=int, default=600, help="frames per stream of the paced latency run (0: skip)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,271 @@
+/*
+ * tt.h — C ABI of the B200-native per-frame hot path for K concurrent tool-tracking streams.
+ *
+ * Problem statement (paper, Sections I and V-B): N identical applications run at once,
+ * each consuming its own frame stream through a recurrent model and producing per-frame
+ * tracking output under an end-to-end latency budget.  Here the N applications become K
+ * stream slots of one context on one GPU; every tick the K frames are batched into one
+ * sequence of launches so that per-frame latency stays flat as K grows.
+ *
+ * The per-frame operator chain is the one of the paper's Endoscopy Tool Tracking
+ * application (Section III-A): format conversion -> recurrent (LSTM) inference ->
+ * tool-tracking post-processing -> overlay.  The paper does not give the arithmetic of
+ * these operators; the definitions are stated with each call below.
+ *
+ * Conventions
+ *   - plain C99 types only; every call returns tt_status and never aborts or throws;
+ *   - "host" / "device" is stated for every pointer; device pointers must belong to the
+ *     context's CUDA device;
+ *   - all work is enqueued on the context's CUDA stream (paper Section III-A: one stream
+ *     is allocated at format conversion and reused by the operators after it);
+ *   - no entry point has a CPU fallback: without a usable sm_100 device calls fail with
+ *     TT_ERR_CUDA / TT_ERR_UNSUPPORTED.
+ */
+#ifndef TT_H_
+#define TT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TT_ABI_VERSION 1u
+#define TT_MAX_STREAMS 8
+#define TT_MAX_TOOLS 8
+#define TT_MAX_ENC 4
+
+typedef enum {
+  TT_OK = 0,
+  TT_ERR_INVALID_ARG = 1,   /* null pointer, bad size, duplicate state, wrong struct_size */
+  TT_ERR_UNSUPPORTED = 2,   /* shape / precision combination the kernels do not cover */
+  TT_ERR_OOM = 3,           /* device or host allocation failed */
+  TT_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed; see tt_last_error */
+  TT_ERR_ADMISSION = 5,     /* more streams than the context was sized for (Section IV-A, admission control) */
+  TT_ERR_NOT_READY = 6,     /* submit while a submit is in flight, or sync with nothing submitted */
+  TT_ERR_TIMEOUT = 7,       /* bounded wait expired; the device is left usable */
+  TT_ERR_DEVICE_STATUS = 8  /* a kernel reported a bounded device-side wait that ran out */
+} tt_status;
+
+typedef enum { TT_FP32 = 0, TT_BF16 = 1 } tt_precision;
+typedef enum { TT_CONF_MEAN_SIGMOID = 0, TT_CONF_GAP_LINEAR = 1 } tt_conf_mode;
+
+/* Which intermediate tensor tt_debug_tensor copies out (always NCHW fp32 on the host). */
+typedef enum {
+  TT_TENSOR_PRE = 0,      /* [3][net_h][net_w]                       */
+  TT_TENSOR_ENC0 = 1,     /* [enc_cout[l]][H_l][W_l], l = which - 1  */
+  TT_TENSOR_ENC1 = 2,
+  TT_TENSOR_ENC2 = 3,
+  TT_TENSOR_ENC3 = 4,
+  TT_TENSOR_H = 8,        /* [hidden][Hm][Wm] state after the last step */
+  TT_TENSOR_C = 9,
+  TT_TENSOR_LOGITS = 10,  /* [n_tools][Hm][Wm] */
+  TT_TENSOR_PROB = 11     /* [n_tools][Hm][Wm] */
+} tt_tensor_id;
+
+typedef struct {
+  uint32_t struct_size;            /* = sizeof(tt_config) */
+  uint32_t abi_version;            /* = TT_ABI_VERSION */
+  int32_t device;                  /* CUDA device ordinal */
+  int32_t max_streams;             /* K_max, 1..TT_MAX_STREAMS; also the number of state slots */
+  int32_t src_w, src_h, src_pitch; /* uint8 RGB interleaved frames, pitch in bytes >= 3*src_w */
+  int32_t net_w, net_h;            /* resize target */
+  float norm_div, norm_mean, norm_std; /* out = ((v / div) - mean) / std */
+  int32_t n_enc;                   /* 1..TT_MAX_ENC encoder layers: 3x3 conv, pad 1, bias, ReLU */
+  int32_t enc_cout[TT_MAX_ENC];
+  int32_t enc_stride[TT_MAX_ENC];  /* 1 or 2 */
+  int32_t hidden;                  /* ConvLSTM hidden channels; 3x3, stride 1, pad 1 */
+  int32_t n_tools;                 /* 1..TT_MAX_TOOLS */
+  int32_t precision;               /* tt_precision */
+  int32_t conf_mode;               /* tt_conf_mode */
+  float threshold;                 /* on the sigmoid, in (0,1) */
+  int32_t overlay;                 /* non-zero: also produce the RGBA8 overlay per frame */
+  uint8_t palette[TT_MAX_TOOLS][3];
+  uint8_t reserved_[8];
+  void* cuda_stream;               /* cudaStream_t owned by the caller, or NULL: the library creates one */
+  uint64_t sync_timeout_ns;        /* 0: wait without limit in tt_sync */
+} tt_config;
+
+/* Host pointers, fp32, framework-conventional layouts.  Copied and repacked by tt_create;
+ * the caller may free them afterwards.  On a TT_BF16 context every weight tensor is
+ * rounded to bf16 (nearest even) while repacking; biases stay fp32. */
+typedef struct {
+  const float* enc_w[TT_MAX_ENC];  /* [Cout][Cin][3][3] */
+  const float* enc_b[TT_MAX_ENC];  /* [Cout] */
+  const float* lstm_w;             /* [4*hidden][Cx+hidden][3][3]; output blocks i|f|g|o, input channels x then h */
+  const float* lstm_b;             /* [4*hidden] */
+  const float* head_w;             /* [n_tools][hidden] */
+  const float* head_b;             /* [n_tools] */
+  const float* conf_w;             /* [n_tools][hidden]; NULL for TT_CONF_MEAN_SIGMOID */
+  const float* conf_b;             /* [n_tools] */
+} tt_weights;
+
+typedef struct tt_ctx tt_ctx;     /* opaque, library-owned */
+typedef struct tt_state tt_state; /* opaque recurrent state (h, c) of one stream, owned by its context */
+
+typedef struct {
+  const uint8_t* data;   /* [src_h][src_pitch] bytes; device memory if on_device != 0, else pinned host memory */
+  int32_t on_device;
+  int32_t reserved_;
+  uint64_t frame_index;  /* echoed into the result */
+  uint64_t arrival_ns;   /* caller's clock; echoed, not interpreted */
+} tt_frame;
+
+typedef struct {
+  uint64_t frame_index;
+  uint64_t arrival_ns;
+  float conf[TT_MAX_TOOLS];
+  float cx[TT_MAX_TOOLS];      /* mask centroid in mask-grid index coordinates; -1 when the mask is empty */
+  float cy[TT_MAX_TOOLS];
+  int32_t count[TT_MAX_TOOLS]; /* pixels above threshold */
+  const uint8_t* masks_dev;    /* device, [n_tools][Hm][Wm] 0/1; valid until the next submit */
+  const float* probs_dev;      /* device, [n_tools][Hm][Wm]; valid until the next submit */
+  const uint8_t* overlay_dev;  /* device, [src_h][src_w][4] RGBA8, or NULL when overlay is off */
+  float gpu_ms;                /* device time of the whole batch this frame was part of */
+  int32_t reserved_;
+} tt_result;
+
+uint32_t tt_abi_version(void);
+
+/*
+ * tt_create — build a context for one model and up to max_streams concurrent streams
+ * (the paper's N concurrent application instances, Section V-B, all running the same
+ * model).  Validates the configuration, allocates every activation, state and output
+ * buffer for max_streams on cfg->device, repacks the weights into the kernels' internal
+ * layouts and builds the TMA tensor maps.  On error *out is NULL; tt_last_error(NULL)
+ * describes a failed create.
+ */
+tt_status tt_create(const tt_config* cfg, const tt_weights* weights, tt_ctx** out);
+
+/* Frees everything the context owns, states included.  NULL is accepted. */
+tt_status tt_destroy(tt_ctx* ctx);
+
+/* Last error text of the context (or of the last failed tt_create when ctx is NULL).
+ * The pointer stays valid until the next failing call on the same context. */
+const char* tt_last_error(const tt_ctx* ctx);
+
+/* Mask-grid (= encoder output = recurrent state) extent of the context. */
+tt_status tt_map_size(const tt_ctx* ctx, int32_t* hm, int32_t* wm);
+
+/*
+ * Recurrent state of one stream.  The paper keeps it inside the inference operator
+ * (Section III-A); here it is an explicit object so that streams can be reset, exported
+ * and re-imported.  A context holds at most max_streams states (TT_ERR_ADMISSION beyond).
+ * create/reset zero h and c.  export/import use host fp32 buffers [hidden][Hm][Wm]
+ * (NCHW) and are synchronous with the context's stream.
+ */
+tt_status tt_state_create(tt_ctx* ctx, tt_state** out);
+tt_status tt_state_reset(tt_ctx* ctx, tt_state* st);
+tt_status tt_state_export(tt_ctx* ctx, tt_state* st, float* h_host, float* c_host);
+tt_status tt_state_import(tt_ctx* ctx, tt_state* st, const float* h_host, const float* c_host);
+
+/*
+ * tt_submit_frames — enqueue one tick: the newest frame of K streams, each with its own
+ * recurrent state, goes through the whole per-frame chain (Section III-A):
+ *   S1 preprocess   bilinear resize (half-pixel centres, edge clamp, no antialias) of the
+ *                   uint8 RGB frame to net_w x net_h, normalise, planar fp32;
+ *   S2 encoder      n_enc x [3x3 conv, pad 1, stride enc_stride[l], bias, ReLU];
+ *   S3 ConvLSTM     gates = W (*) concat[x, h] + b; c' = s(f) c + s(i) tanh(g); h' = s(o) tanh(c');
+ *   S4 mask head    z = 1x1 conv(h') + b; p = sigmoid(z); mask = z > logit(threshold);
+ *   S5 per tool     confidence (mean of p, or sigmoid(linear(global-average-pool(h')))),
+ *                   count and centroid of the mask;
+ *   S6 overlay      (if enabled) alpha-0.4 integer blend of the masks onto an RGBA8 copy.
+ * Asynchronous: returns once the work is enqueued.  frames[k].data must stay valid until
+ * tt_sync returns.  Errors: K < 1 or null/duplicate/foreign states -> TT_ERR_INVALID_ARG;
+ * K > max_streams -> TT_ERR_ADMISSION; a submit already in flight -> TT_ERR_NOT_READY.
+ * Nothing is enqueued when one of these argument errors is returned.
+ */
+tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_state* const* states);
+
+/*
+ * tt_sync — wait for the submit in flight and fill results[0..K-1] (host, caller-owned,
+ * same order as the submitted frames).  This is the "departure from the leaf operator" of
+ * the paper's end-to-end latency definition (Section II-C).  With a non-zero
+ * sync_timeout_ns the wait is bounded: TT_ERR_TIMEOUT leaves the submit in flight and the
+ * call may be repeated.  TT_ERR_DEVICE_STATUS: a kernel gave up a bounded device-side
+ * wait; results are invalid, the context stays usable.
+ */
+tt_status tt_sync(tt_ctx* ctx, tt_result* results);
+
+/*
+ * tt_debug_tensor — copy one intermediate tensor of the last completed submit for the
+ * stream that used `st` into host_dst as NCHW fp32 (cap = capacity in floats).
+ * Synchronous; for tests and parity checks only.
+ */
+tt_status tt_debug_tensor(tt_ctx* ctx, tt_state* st, int32_t which, float* host_dst, size_t cap);
+
+/*
+ * Measurement hooks (the paper times every operator's input and output, Section II-C, data
+ * flow tracking; here CUDA events on the context's stream bracket each stage of a tick).
+ * tt_set_profiling(on != 0) makes every following submit record stage events.
+ * tt_get_stage_times fills ms[TT_STAGE_COUNT] (host) with the device time of each stage of
+ * the last completed submit, -1 for stages that did not run or when profiling was off.
+ * tt_get_counters reports how many of the library's kernels and ticks this context has
+ * launched since creation.
+ */
+typedef enum {
+  TT_STAGE_H2D = 0,        /* host->device frame copies (frames with on_device == 0) */
+  TT_STAGE_PREPROCESS = 1,
+  TT_STAGE_ENC0 = 2,       /* encoder layer l = stage 2 + l */
+  TT_STAGE_ENC1 = 3,
+  TT_STAGE_ENC2 = 4,
+  TT_STAGE_ENC3 = 5,
+  TT_STAGE_CONVLSTM = 6,
+  TT_STAGE_POSTPROCESS = 7,
+  TT_STAGE_OVERLAY = 8,
+  TT_STAGE_COUNT = 9
+} tt_stage;
+tt_status tt_set_profiling(tt_ctx* ctx, int32_t on);
+tt_status tt_get_stage_times(tt_ctx* ctx, float* ms);
+tt_status tt_get_counters(const tt_ctx* ctx, uint64_t* kernel_launches, uint64_t* ticks);
+
+/* ---------------------------------------------------------------------------------------
+ * Stage-level entry points on caller-owned device buffers (no context needed).  They run
+ * the same kernels as the corresponding stage of tt_submit_frames and are asynchronous on
+ * `cuda_stream` (a cudaStream_t, NULL = default stream).
+ * ------------------------------------------------------------------------------------ */
+
+/*
+ * tt_preprocess — S1, the format-conversion operator of Section III-A.
+ * src_dev: K frames, frame k at src_dev + k*src_frame_stride bytes, uint8 RGB interleaved,
+ * row pitch src_pitch bytes.  dst_dev: fp32 [K][3][net_h][net_w].  For output sample o of
+ * an axis resized from `in` to `out`: s = clamp((o+1/2)*in/out - 1/2, 0, in-1) evaluated in
+ * exact integer arithmetic, i0 = floor(s), i1 = min(i0+1, in-1), weight s - i0.
+ */
+tt_status tt_preprocess(const uint8_t* src_dev, int32_t K, int64_t src_frame_stride, int32_t src_w,
+                        int32_t src_h, int32_t src_pitch, float* dst_dev, int32_t net_w, int32_t net_h,
+                        float norm_div, float norm_mean, float norm_std, void* cuda_stream);
+
+/*
+ * tt_postprocess — S4+S5, the tool-tracking post-processing operator of Section III-A.
+ * h_dev: fp32 hidden state of K streams, channels-last [K][Hm][Wm][hidden] when
+ * channels_last != 0, else planar [K][hidden][Hm][Wm].  head_w/head_b (and conf_w/conf_b
+ * for TT_CONF_GAP_LINEAR) are device fp32 [n_tools][hidden] / [n_tools].
+ * Outputs (device): logits, probs fp32 [K][n_tools][Hm][Wm]; masks uint8 same shape;
+ * results: K tt_result records of which conf, cx, cy, count are written.
+ * scratch_dev: tt_postprocess_scratch_bytes(...) bytes of device memory, contents ignored.
+ * hidden must be a multiple of 4 and at most 512.
+ */
+size_t tt_postprocess_scratch_bytes(int32_t K, int32_t hm, int32_t wm, int32_t hidden, int32_t n_tools);
+tt_status tt_postprocess(const float* h_dev, int32_t channels_last, int32_t K, int32_t hm, int32_t wm,
+                         int32_t hidden, int32_t n_tools, const float* head_w_dev, const float* head_b_dev,
+                         const float* conf_w_dev, const float* conf_b_dev, int32_t conf_mode, float threshold,
+                         float* logits_dev, float* probs_dev, uint8_t* masks_dev, tt_result* results_dev,
+                         void* scratch_dev, void* cuda_stream);
+
+/*
+ * tt_overlay — S6, the stand-in for the visualisation operator of Section II-B / III-A
+ * (mask overlay on the frame).  src_dev as in tt_preprocess; masks_dev uint8
+ * [K][n_tools][Hm][Wm]; palette: n_tools RGB triples (host); dst_dev uint8
+ * [K][src_h][src_w][4].  Mask sample for source pixel (x, y): (floor(x*Wm/src_w),
+ * floor(y*Hm/src_h)); tools blended in ascending order as (153*rgb + 102*colour + 127)/255.
+ */
+tt_status tt_overlay(const uint8_t* src_dev, int32_t K, int64_t src_frame_stride, int32_t src_w, int32_t src_h,
+                     int32_t src_pitch, const uint8_t* masks_dev, int32_t n_tools, int32_t hm, int32_t wm,
+                     const uint8_t* palette_host, uint8_t* dst_dev, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TT_H_ */

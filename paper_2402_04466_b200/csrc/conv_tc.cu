@@ -1,0 +1,415 @@
+// S2/S3 on the 5th-generation tensor cores: 3x3 convolution (pad 1, stride 1 or 2) as an
+// implicit GEMM.  M = output pixels (a 16 x 8 patch = 128 rows per tile), N = output
+// channels, K = 9 taps x input channels.  No im2col buffer exists anywhere: for every tap
+// the producer issues one 4-D TMA box load of the shifted activation patch (NHWC bf16,
+// 128-byte or 64-byte swizzle, out-of-range rows and columns zero-filled by the TMA unit,
+// which is exactly the convolution's zero padding) and one 2-D TMA load of the matching
+// K-slab of the packed weights.  tcgen05.mma accumulates in TMEM; two accumulator buffers
+// let the epilogue of tile i overlap the main loop of tile i+1.  The epilogue reads TMEM
+// with tcgen05.ld and applies bias + ReLU (encoder) or the whole ConvLSTM gate math
+// (sigmoid/tanh, c' = f*c + i*g, h' = o*tanh(c')) so gate pre-activations never reach HBM.
+//
+// Stride-2 layers read four "parity views" of their input (even/odd rows x even/odd
+// columns), each an ordinary tiled tensor map with doubled strides, so every tap is again
+// a dense box.
+//
+// Warp roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM allocation and
+// MMA issue (one lane), warps 2..5 = epilogue (TMEM lane quarter = warp index mod 4).
+// Every mbarrier wait is bounded: when a wait runs out the kernel records a status code,
+// raises a block-wide abort flag, lets copies in flight land, frees its TMEM and returns.
+#include "tt_internal.h"
+
+namespace tt {
+namespace {
+
+constexpr int BLOCK_M = 128;
+constexpr int PATCH_W = 16, PATCH_H = 8;
+constexpr int UMMA_K = 16;
+constexpr int TC_THREADS = 192;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s per wait
+
+template <int BLOCK_N, int SLAB_C>
+struct TcCfg {
+  static constexpr int A_BYTES = BLOCK_M * SLAB_C * 2;
+  static constexpr int B_BYTES = BLOCK_N * SLAB_C * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES_RAW = (192 * 1024) / STAGE_BYTES;
+  static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
+  static constexpr int TMEM_COLS = 2 * BLOCK_N < 32 ? 32 : 2 * BLOCK_N;
+  static constexpr int BAR_BYTES = 256;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024 /*alignment slack*/;
+  static_assert((TMEM_COLS & (TMEM_COLS - 1)) == 0 && TMEM_COLS <= 512, "TMEM columns must be a power of two <= 512");
+  static_assert(A_BYTES % 1024 == 0 && B_BYTES % 1024 == 0, "operand tiles must keep 1024-byte alignment");
+};
+
+// ------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait.  Returns false when the block is aborting (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 31u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// K-major operand tile in shared memory: rows of SLAB_C bf16 (128 or 64 bytes), swizzled in
+// atoms of 8 rows; consecutive 8-row groups are SBO = 8 * row bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t sbo_bytes, uint32_t layout_type) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                           // leading byte offset: unused for swizzled K-major
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;  // stride byte offset
+  d |= (uint64_t)1 << 46;                           // descriptor version of this architecture
+  d |= (uint64_t)layout_type << 61;                 // 2 = 128-byte swizzle, 4 = 64-byte swizzle
+  return d;
+}
+
+// kind::f16 instruction descriptor: D = fp32, A = B = bf16, both K-major, M x N tile.
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ float fast_sigmoid(float z) { return __frcp_rn(1.0f + __expf(-z)); }
+__device__ __forceinline__ float fast_tanh(float z) { return 1.0f - 2.0f * __frcp_rn(1.0f + __expf(2.0f * z)); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ------------------------------------------------------------------------------------ kernel
+template <int BLOCK_N, int SLAB_C, int EPI>
+__global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_constant__ ConvTcParams p) {
+  using Cfg = TcCfg<BLOCK_N, SLAB_C>;
+  constexpr int STAGES = Cfg::STAGES;
+  constexpr uint32_t LAYOUT = SLAB_C == 64 ? 2u : 4u;
+  constexpr uint32_t SBO = 8u * SLAB_C * 2u;
+  constexpr uint32_t IDESC = make_idesc(BLOCK_M, BLOCK_N);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* bar_mem = smem + STAGES * Cfg::STAGE_BYTES;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(bar_mem);   // [STAGES]
+  uint64_t* empty_bar = full_bar + STAGES;                     // [STAGES]
+  uint64_t* tfull_bar = empty_bar + STAGES;                    // [2]
+  uint64_t* tempty_bar = tfull_bar + 2;                        // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(full_bar + s), 1);
+      mbar_init(smem_u32(empty_bar + s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(tfull_bar + a), 1);
+      mbar_init(smem_u32(tempty_bar + a), 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)Cfg::TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_per_img = p.tiles_x * p.tiles_y;
+  const int total_tiles = p.K * tiles_per_img * p.n_tiles_n;
+  const int slabs_per_tap = p.slabs[0] + (p.n_src > 1 ? p.slabs[1] : 0);
+  const int k_iters = 9 * slabs_per_tap;
+
+  if (warp == 0 && lane == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    uint32_t stage = 0, phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int nt = tile % p.n_tiles_n;
+      const int m = tile / p.n_tiles_n;
+      const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
+      const int x0 = tx * PATCH_W, y0 = ty * PATCH_H;
+      int kcol = 0;
+      for (int tap = 0; tap < 9 && ok; ++tap) {
+        const int ky = tap / 3, kx = tap % 3;
+        int cx, cy, par;
+        if (p.stride == 1) {
+          cx = x0 + kx - 1;
+          cy = y0 + ky - 1;
+          par = 0;
+        } else {
+          // input column 2*xo + kx - 1: kx = 1 is the even view at xo, kx = 0 / 2 the odd view at xo-1 / xo
+          const int xpar = (kx == 1) ? 0 : 1, ypar = (ky == 1) ? 0 : 1;
+          cx = x0 + (kx == 0 ? -1 : 0);
+          cy = y0 + (ky == 0 ? -1 : 0);
+          par = ypar * 2 + xpar;
+        }
+        for (int src = 0; src < p.n_src && ok; ++src) {
+          const void* map_a = &p.maps_a[src * 4 + par];
+          const int img_idx = src == 0 ? p.img0.v[img] : p.img1.v[img];
+          for (int sl = 0; sl < p.slabs[src]; ++sl) {
+            ok = mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag, p.status, 0x100 + (int)stage);
+            if (!ok) break;
+            const uint32_t fb = smem_u32(full_bar + stage);
+            uint8_t* st = smem + stage * Cfg::STAGE_BYTES;
+            mbar_arrive_expect_tx(fb, Cfg::STAGE_BYTES);
+            tma_load_4d(smem_u32(st), map_a, fb, sl * SLAB_C, cx, cy, img_idx);
+            tma_load_2d(smem_u32(st + Cfg::A_BYTES), &p.map_b, fb, kcol, nt * BLOCK_N);
+            kcol += SLAB_C;
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // -------------------------------------------------------------------- MMA issuer
+    uint32_t stage = 0, phase = 0, acc_phase = 0;
+    int acc = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      ok = mbar_wait(smem_u32(tempty_bar + acc), acc_phase ^ 1u, abort_flag, p.status, 0x200 + acc);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BLOCK_N);
+      for (int it = 0; it < k_iters; ++it) {
+        ok = mbar_wait(smem_u32(full_bar + stage), phase, abort_flag, p.status, 0x300 + (int)stage);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(smem + stage * Cfg::STAGE_BYTES);
+        const uint32_t b_addr = a_addr + Cfg::A_BYTES;
+        const uint64_t a_desc = make_smem_desc(a_addr, SBO, LAYOUT);
+        const uint64_t b_desc = make_smem_desc(b_addr, SBO, LAYOUT);
+#pragma unroll
+        for (int k = 0; k < SLAB_C / UMMA_K; ++k) {
+          // advance along K inside the swizzle atom: 16 bf16 = 32 bytes = 2 descriptor units
+          umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), IDESC, (it | k) != 0 ? 1u : 0u);
+        }
+        umma_commit(smem_u32(empty_bar + stage));  // frees the stage once the MMAs have read it
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) break;
+      umma_commit(smem_u32(tfull_bar + acc));      // accumulator complete
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  } else if (warp >= 2) {
+    // ---------------------------------------------------------------------- epilogue
+    const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
+    const int row = quarter * 32 + lane;          // row of the 128-row tile = pixel of the patch
+    const int py = row / PATCH_W, px = row % PATCH_W;
+    uint32_t acc_phase = 0;
+    int acc = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const int nt = tile % p.n_tiles_n;
+      const int m = tile / p.n_tiles_n;
+      const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
+      const int x = tx * PATCH_W + px, y = ty * PATCH_H + py;
+      const bool valid = x < p.Wo && y < p.Ho;
+      ok = mbar_wait(smem_u32(tfull_bar + acc), acc_phase, abort_flag, p.status, 0x400 + acc);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
+      const size_t pix = (size_t)y * p.Wo + x;
+#pragma unroll 1
+      for (int ch0 = 0; ch0 < BLOCK_N; ch0 += 32) {
+        uint32_t v[32];
+        tmem_ld32(t_addr + (uint32_t)ch0, v);
+        const int n0 = nt * BLOCK_N + ch0;        // first packed output column of this chunk
+        if (EPI == TC_EPI_RELU_BF16) {
+          if (valid && n0 < p.cout) {
+            const float4* b4 = reinterpret_cast<const float4*>(p.bias + n0);
+            __nv_bfloat16* dst = p.out + ((size_t)img * p.Ho * p.Wo + pix) * p.cout + n0;
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              const float4 ba = __ldg(b4 + i / 4), bb = __ldg(b4 + i / 4 + 1);
+              uint4 u;
+              u.x = pack_bf16(fmaxf(__uint_as_float(v[i + 0]) + ba.x, 0.f), fmaxf(__uint_as_float(v[i + 1]) + ba.y, 0.f));
+              u.y = pack_bf16(fmaxf(__uint_as_float(v[i + 2]) + ba.z, 0.f), fmaxf(__uint_as_float(v[i + 3]) + ba.w, 0.f));
+              u.z = pack_bf16(fmaxf(__uint_as_float(v[i + 4]) + bb.x, 0.f), fmaxf(__uint_as_float(v[i + 5]) + bb.y, 0.f));
+              u.w = pack_bf16(fmaxf(__uint_as_float(v[i + 6]) + bb.z, 0.f), fmaxf(__uint_as_float(v[i + 7]) + bb.w, 0.f));
+              *reinterpret_cast<uint4*>(dst + i) = u;
+            }
+          }
+        } else {
+          // packed column = 4*jj + gate (i, f, g, o); 8 hidden units per 32-column chunk
+          const int j0 = n0 >> 2;
+          if (valid && j0 < p.hidden) {
+            const float4* b4 = reinterpret_cast<const float4*>(p.bias + n0);
+            const size_t so = ((size_t)p.c_idx.v[img] * p.Ho * p.Wo + pix) * p.hidden + j0;
+            const size_t ho = ((size_t)p.h_out_idx.v[img] * p.Ho * p.Wo + pix) * p.hidden + j0;
+            float* c_ptr = p.c_state + so;
+            float* h_ptr = p.h_f32 + so;
+            const float4 c_lo = *reinterpret_cast<const float4*>(c_ptr);
+            const float4 c_hi = *reinterpret_cast<const float4*>(c_ptr + 4);
+            const float c_old[8] = {c_lo.x, c_lo.y, c_lo.z, c_lo.w, c_hi.x, c_hi.y, c_hi.z, c_hi.w};
+            float c_new[8], h_new[8];
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) {
+              const float4 b = __ldg(b4 + jj);
+              const float gi = __uint_as_float(v[4 * jj + 0]) + b.x;
+              const float gf = __uint_as_float(v[4 * jj + 1]) + b.y;
+              const float gg = __uint_as_float(v[4 * jj + 2]) + b.z;
+              const float go = __uint_as_float(v[4 * jj + 3]) + b.w;
+              c_new[jj] = fast_sigmoid(gf) * c_old[jj] + fast_sigmoid(gi) * fast_tanh(gg);
+              h_new[jj] = fast_sigmoid(go) * fast_tanh(c_new[jj]);
+            }
+            *reinterpret_cast<float4*>(c_ptr) = make_float4(c_new[0], c_new[1], c_new[2], c_new[3]);
+            *reinterpret_cast<float4*>(c_ptr + 4) = make_float4(c_new[4], c_new[5], c_new[6], c_new[7]);
+            *reinterpret_cast<float4*>(h_ptr) = make_float4(h_new[0], h_new[1], h_new[2], h_new[3]);
+            *reinterpret_cast<float4*>(h_ptr + 4) = make_float4(h_new[4], h_new[5], h_new[6], h_new[7]);
+            uint4 hb;
+            hb.x = pack_bf16(h_new[0], h_new[1]);
+            hb.y = pack_bf16(h_new[2], h_new[3]);
+            hb.z = pack_bf16(h_new[4], h_new[5]);
+            hb.w = pack_bf16(h_new[6], h_new[7]);
+            *reinterpret_cast<uint4*>(p.h_bf16 + ho) = hb;
+          }
+        }
+      }
+      // hand the accumulator buffer back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(tempty_bar + acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ------------------------------------------------------------------------------- teardown
+  __syncwarp();
+  if (*abort_flag) {
+    // a wait ran out somewhere: give copies and MMAs in flight time to land before the
+    // shared memory and TMEM of this block are released
+    for (int i = 0; i < 64; ++i) __nanosleep(16000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS)
+                 : "memory");
+  }
+}
+
+template <int BLOCK_N, int SLAB_C, int EPI>
+cudaError_t launch_cfg(const ConvTcParams& p, int sm_count, cudaStream_t s) {
+  using Cfg = TcCfg<BLOCK_N, SLAB_C>;
+  auto kern = conv_tc_kernel<BLOCK_N, SLAB_C, EPI>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  const int total_tiles = p.K * p.tiles_x * p.tiles_y * p.n_tiles_n;
+  const int grid = total_tiles < sm_count ? total_tiles : sm_count;
+  kern<<<grid, TC_THREADS, Cfg::SMEM_BYTES, s>>>(p);
+  return cudaGetLastError();
+}
+
+template <int EPI>
+cudaError_t launch_shape(const ConvTcParams& p, int sm_count, cudaStream_t s) {
+  if (p.slab_c == 64) {
+    if (p.block_n == 256) return launch_cfg<256, 64, EPI>(p, sm_count, s);
+    if (p.block_n == 128) return launch_cfg<128, 64, EPI>(p, sm_count, s);
+    if (p.block_n == 64) return launch_cfg<64, 64, EPI>(p, sm_count, s);
+  } else if (p.slab_c == 32) {
+    if (p.block_n == 128) return launch_cfg<128, 32, EPI>(p, sm_count, s);
+    if (p.block_n == 64) return launch_cfg<64, 32, EPI>(p, sm_count, s);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace
+
+cudaError_t conv_tc_prepare() { return cudaSuccess; }
+
+cudaError_t launch_conv_tc(const ConvTcParams& p, int sm_count, cudaStream_t s) {
+  if (p.epilogue == TC_EPI_RELU_BF16) return launch_shape<TC_EPI_RELU_BF16>(p, sm_count, s);
+  if (p.epilogue == TC_EPI_LSTM) return launch_shape<TC_EPI_LSTM>(p, sm_count, s);
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace tt

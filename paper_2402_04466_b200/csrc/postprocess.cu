@@ -1,0 +1,241 @@
+// S4 + S5: mask head (1x1 conv hidden -> tools), sigmoid, threshold, per-tool confidence
+// and mask centroid.  HBM-bound: the hidden state is read exactly once.
+//
+// Pass 1 (post_tile_kernel): a block stages 64 pixels x Ch hidden values in shared memory
+// with coalesced 128-bit loads, four threads per pixel form the T dot products, the masks,
+// logits and probabilities are written, and the block's partial sums (count, sum x, sum y
+// as integers; sum p and per-channel sum h as floats) are written to scratch.
+// Pass 2 (post_finalize_kernel): one block per stream adds the partials in a fixed order
+// (bitwise reproducible, no float atomics) and forms confidence and centroid.
+#include "tt_internal.h"
+
+namespace tt {
+namespace {
+
+constexpr int PIX = 64;        // pixels per block
+constexpr int POST_THREADS = 256;
+constexpr int ROW_PAD = 16;    // floats of padding per staged pixel row
+
+__host__ __device__ inline int post_blocks_per_img(int plane) { return (plane + PIX - 1) / PIX; }
+
+struct ScratchLayout {
+  size_t off_int, off_p, off_h, total;
+};
+__host__ __device__ inline ScratchLayout scratch_layout(int K, int plane, int ch, int T) {
+  const size_t nb = (size_t)K * post_blocks_per_img(plane);
+  ScratchLayout l;
+  l.off_int = 0;
+  l.off_p = l.off_int + nb * TT_MAX_TOOLS * 4 * sizeof(int32_t);
+  l.off_h = l.off_p + nb * TT_MAX_TOOLS * sizeof(float);
+  l.total = l.off_h + nb * (size_t)ch * sizeof(float);
+  l.total = (l.total + 255) & ~(size_t)255;
+  return l;
+}
+
+__device__ __forceinline__ float sigmoid_acc(float z) { return 1.0f / (1.0f + expf(-z)); }
+
+__global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const PostParams p) {
+  extern __shared__ __align__(16) float s_mem[];
+  const int Ch = p.Ch, T = p.T;
+  const int row = Ch + ROW_PAD;
+  float* s_tile = s_mem;                     // [PIX][row]
+  float* s_w = s_tile + PIX * row;           // [T][Ch]
+  float* s_red_f = s_w + TT_MAX_TOOLS * Ch;  // [8 warps][T]
+  int* s_red_i = reinterpret_cast<int*>(s_red_f + 8 * TT_MAX_TOOLS);  // [8 warps][T][3]
+
+  const int plane = p.Hm * p.Wm;
+  const int nb = post_blocks_per_img(plane);
+  const int n = blockIdx.x / nb, blk = blockIdx.x % nb;
+  const int pix0 = blk * PIX;
+  const int npix = min(PIX, plane - pix0);
+  const int tid = threadIdx.x;
+  const float* h_img = p.h + (size_t)p.idx.v[n] * p.img_stride;
+
+  for (int i = tid; i < T * Ch; i += POST_THREADS) s_w[i] = __ldg(p.head_w + i);
+
+  if (p.channels_last) {
+    const int row4 = Ch >> 2;
+    const float4* g = reinterpret_cast<const float4*>(h_img + (size_t)pix0 * Ch);
+    for (int i = tid; i < npix * row4; i += POST_THREADS) {
+      const int pp = i / row4, c4 = i % row4;
+      *reinterpret_cast<float4*>(s_tile + pp * row + 4 * c4) = __ldg(g + i);
+    }
+  } else {
+    for (int i = tid; i < Ch * PIX; i += POST_THREADS) {
+      const int c = i / PIX, pp = i % PIX;
+      if (pp < npix) s_tile[pp * row + c] = __ldg(h_img + (size_t)c * plane + pix0 + pp);
+    }
+  }
+  __syncthreads();
+
+  // --- T dot products per pixel: 4 threads per pixel, 128-bit chunks interleaved by q.
+  const int pp = tid >> 2, q = tid & 3;
+  float acc[TT_MAX_TOOLS];
+#pragma unroll
+  for (int t = 0; t < TT_MAX_TOOLS; ++t) acc[t] = 0.0f;
+  if (pp < npix) {
+    for (int c4 = q; c4 < (Ch >> 2); c4 += 4) {
+      const float4 hv = *reinterpret_cast<const float4*>(s_tile + pp * row + 4 * c4);
+#pragma unroll
+      for (int t = 0; t < TT_MAX_TOOLS; ++t) {
+        if (t < T) {
+          const float4 wv = *reinterpret_cast<const float4*>(s_w + t * Ch + 4 * c4);
+          acc[t] = fmaf(hv.x, wv.x, acc[t]);
+          acc[t] = fmaf(hv.y, wv.y, acc[t]);
+          acc[t] = fmaf(hv.z, wv.z, acc[t]);
+          acc[t] = fmaf(hv.w, wv.w, acc[t]);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int t = 0; t < TT_MAX_TOOLS; ++t) {
+    acc[t] += __shfl_xor_sync(0xffffffffu, acc[t], 1);
+    acc[t] += __shfl_xor_sync(0xffffffffu, acc[t], 2);
+  }
+
+  // --- sigmoid, threshold, outputs, per-pixel statistics (lanes with q == 0 own a pixel)
+  const bool owner = (q == 0) && (pp < npix);
+  const int pix = pix0 + pp;
+  const int px = owner ? pix % p.Wm : 0, py = owner ? pix / p.Wm : 0;
+  uint32_t bits = 0;
+  float prob[TT_MAX_TOOLS];
+#pragma unroll
+  for (int t = 0; t < TT_MAX_TOOLS; ++t) {
+    prob[t] = 0.0f;
+    if (t < T && owner) {
+      const float z = acc[t] + __ldg(p.head_b + t);
+      const float pr = sigmoid_acc(z);
+      const bool m = z > p.zthr;
+      prob[t] = pr;
+      bits |= (m ? 1u : 0u) << t;
+      const size_t o = ((size_t)n * T + t) * plane + pix;
+      p.logits[o] = z;
+      p.probs[o] = pr;
+      p.masks[o] = m ? 1 : 0;
+    }
+  }
+  if (owner && p.bits) p.bits[(size_t)n * plane + pix] = (uint8_t)bits;
+
+  // --- block partial sums: shuffle over the 8 pixel owners of a warp, then over 8 warps
+  const int warp = tid >> 5, lane = tid & 31;
+#pragma unroll
+  for (int t = 0; t < TT_MAX_TOOLS; ++t) {
+    if (t < T) {
+      int cnt = (bits >> t) & 1u;
+      int sx = cnt ? px : 0, sy = cnt ? py : 0;
+      float sp = prob[t];
+#pragma unroll
+      for (int d = 4; d < 32; d <<= 1) {
+        cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+        sx += __shfl_xor_sync(0xffffffffu, sx, d);
+        sy += __shfl_xor_sync(0xffffffffu, sy, d);
+        sp += __shfl_xor_sync(0xffffffffu, sp, d);
+      }
+      if (lane == 0) {
+        s_red_i[(warp * TT_MAX_TOOLS + t) * 3 + 0] = cnt;
+        s_red_i[(warp * TT_MAX_TOOLS + t) * 3 + 1] = sx;
+        s_red_i[(warp * TT_MAX_TOOLS + t) * 3 + 2] = sy;
+        s_red_f[warp * TT_MAX_TOOLS + t] = sp;
+      }
+    }
+  }
+  __syncthreads();
+
+  const ScratchLayout sl = scratch_layout(p.K, plane, Ch, T);
+  uint8_t* scr = reinterpret_cast<uint8_t*>(p.scratch);
+  int32_t* part_i = reinterpret_cast<int32_t*>(scr + sl.off_int) + (size_t)blockIdx.x * TT_MAX_TOOLS * 4;
+  float* part_p = reinterpret_cast<float*>(scr + sl.off_p) + (size_t)blockIdx.x * TT_MAX_TOOLS;
+  float* part_h = reinterpret_cast<float*>(scr + sl.off_h) + (size_t)blockIdx.x * Ch;
+  if (tid < T) {
+    int cnt = 0, sx = 0, sy = 0;
+    float sp = 0.0f;
+    for (int w = 0; w < 8; ++w) {
+      cnt += s_red_i[(w * TT_MAX_TOOLS + tid) * 3 + 0];
+      sx += s_red_i[(w * TT_MAX_TOOLS + tid) * 3 + 1];
+      sy += s_red_i[(w * TT_MAX_TOOLS + tid) * 3 + 2];
+      sp += s_red_f[w * TT_MAX_TOOLS + tid];
+    }
+    part_i[tid * 4 + 0] = cnt;
+    part_i[tid * 4 + 1] = sx;
+    part_i[tid * 4 + 2] = sy;
+    part_p[tid] = sp;
+  }
+  if (p.conf_mode == TT_CONF_GAP_LINEAR) {
+    for (int c = tid; c < Ch; c += POST_THREADS) {
+      float s = 0.0f;
+      for (int i = 0; i < npix; ++i) s += s_tile[i * row + c];
+      part_h[c] = s;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(POST_THREADS) post_finalize_kernel(const PostParams p) {
+  __shared__ float s_gap[512];
+  const int n = blockIdx.x, tid = threadIdx.x;
+  const int plane = p.Hm * p.Wm, Ch = p.Ch, T = p.T;
+  const int nb = post_blocks_per_img(plane);
+  const ScratchLayout sl = scratch_layout(p.K, plane, Ch, T);
+  const uint8_t* scr = reinterpret_cast<const uint8_t*>(p.scratch);
+  const int32_t* part_i = reinterpret_cast<const int32_t*>(scr + sl.off_int) + (size_t)n * nb * TT_MAX_TOOLS * 4;
+  const float* part_p = reinterpret_cast<const float*>(scr + sl.off_p) + (size_t)n * nb * TT_MAX_TOOLS;
+  const float* part_h = reinterpret_cast<const float*>(scr + sl.off_h) + (size_t)n * nb * Ch;
+  const float inv_plane = 1.0f / (float)plane;
+
+  if (p.conf_mode == TT_CONF_GAP_LINEAR) {
+    for (int c = tid; c < Ch; c += POST_THREADS) {
+      float s = 0.0f;
+      for (int b = 0; b < nb; ++b) s += part_h[(size_t)b * Ch + c];
+      s_gap[c] = s * inv_plane;
+    }
+  }
+  __syncthreads();
+  if (tid < T) {
+    long long cnt = 0, sx = 0, sy = 0;
+    float sp = 0.0f;
+    for (int b = 0; b < nb; ++b) {
+      cnt += part_i[((size_t)b * TT_MAX_TOOLS + tid) * 4 + 0];
+      sx += part_i[((size_t)b * TT_MAX_TOOLS + tid) * 4 + 1];
+      sy += part_i[((size_t)b * TT_MAX_TOOLS + tid) * 4 + 2];
+      sp += part_p[(size_t)b * TT_MAX_TOOLS + tid];
+    }
+    float conf;
+    if (p.conf_mode == TT_CONF_GAP_LINEAR) {
+      float a = __ldg(p.conf_b + tid);
+      for (int c = 0; c < Ch; ++c) a = fmaf(__ldg(p.conf_w + tid * Ch + c), s_gap[c], a);
+      conf = sigmoid_acc(a);
+    } else {
+      conf = sp * inv_plane;
+    }
+    tt_result* r = p.results + n;
+    r->conf[tid] = conf;
+    r->count[tid] = (int32_t)cnt;
+    r->cx[tid] = cnt ? (float)((double)sx / (double)cnt) : -1.0f;
+    r->cy[tid] = cnt ? (float)((double)sy / (double)cnt) : -1.0f;
+  }
+}
+
+size_t post_smem_bytes(int ch) {
+  return (size_t)(PIX * (ch + ROW_PAD) + TT_MAX_TOOLS * ch + 8 * TT_MAX_TOOLS) * sizeof(float) +
+         (size_t)8 * TT_MAX_TOOLS * 3 * sizeof(int);
+}
+
+}  // namespace
+
+size_t post_scratch_bytes(int K, int hm, int wm, int ch, int T) { return scratch_layout(K, hm * wm, ch, T).total; }
+
+cudaError_t post_prepare() {
+  return cudaFuncSetAttribute(post_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)post_smem_bytes(512));
+}
+
+cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s) {
+  const int plane = p.Hm * p.Wm;
+  const int nb = post_blocks_per_img(plane);
+  post_tile_kernel<<<p.K * nb, POST_THREADS, post_smem_bytes(p.Ch), s>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  post_finalize_kernel<<<p.K, POST_THREADS, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace tt

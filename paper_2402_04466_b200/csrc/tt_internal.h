@@ -1,0 +1,141 @@
+// Internal launch interfaces shared by the translation units of libtt.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "tt.h"
+
+namespace tt {
+
+// Maps batch position n (0..K-1) of a launch to an image index inside a tensor that holds
+// more images than the batch (state slots, ping-pong halves).
+struct IdxMap {
+  int32_t v[TT_MAX_STREAMS];
+};
+
+struct FramePtrs {
+  const uint8_t* p[TT_MAX_STREAMS];
+};
+
+// ------------------------------------------------------------------------- S1 preprocess
+struct PreprocessParams {
+  FramePtrs src;
+  int32_t K, src_w, src_h, src_pitch, net_w, net_h;
+  float inv_div, mean, inv_std;
+  float* dst;  // [K][3][net_h][net_w]
+};
+cudaError_t launch_preprocess(const PreprocessParams& p, cudaStream_t s);
+
+// ------------------------------------------------------------------ S2/S3 fp32 SIMT conv
+enum ConvEpilogue : int32_t {
+  EPI_RELU_F32_NCHW = 0,   // out fp32 [K][Cout][Ho][Wo]
+  EPI_RELU_BF16_NHWC = 1,  // out bf16 [K][Ho][Wo][Cout]
+  EPI_LSTM_F32_NCHW = 2    // gate math, c in place, h' to the "out" half of the ping-pong
+};
+
+struct ConvSimtParams {
+  const float* in0;  // fp32 planar, image n at in0 + idx0.v[n]*img_stride0
+  const float* in1;  // optional second source (recurrent h), channels follow in0's
+  int64_t img_stride0, img_stride1;
+  IdxMap idx0, idx1;
+  int32_t C0, C1;
+  int32_t H, W, Ho, Wo, stride, K;
+  const float* wgt;   // packed [Cin][9][CoutPacked]
+  const float* bias;  // packed [CoutPacked]
+  int32_t cout, cout_packed, ocb;
+  int32_t epilogue;
+  // EPI_RELU_*: out; EPI_LSTM: c (in place), h_out
+  void* out;
+  int64_t out_img_stride;  // elements
+  float* c_state;          // [slots][Ch][plane]
+  float* h_state;          // [slots*2][Ch][plane]
+  IdxMap c_idx, h_out_idx;
+  int32_t hidden;
+};
+cudaError_t launch_conv_simt(const ConvSimtParams& p, cudaStream_t s);
+
+// ------------------------------------------------- S2/S3 tcgen05 implicit-GEMM conv (bf16)
+// One launch description; tensor maps live in device-visible constant storage owned by the
+// caller (passed by value as __grid_constant__ kernel parameters).
+struct alignas(64) TensorMap128 {
+  uint8_t bytes[128];
+};
+
+enum TcEpilogue : int32_t { TC_EPI_RELU_BF16 = 0, TC_EPI_LSTM = 1 };
+
+struct ConvTcParams {
+  // A operand sources: up to two NHWC bf16 tensors (x then h); for stride 2 four parity
+  // views of the single source.  maps_a[src*4 + parity] with parity = (ypar*2 + xpar).
+  TensorMap128 maps_a[8];
+  TensorMap128 map_b;       // packed weights [CoutPacked][Ktot] bf16, K-major
+  int32_t n_src;            // 1 or 2
+  int32_t slabs[2];         // channel slabs (of slab_c channels) per source
+  int32_t slab_c;           // 64 or 32
+  int32_t stride;           // 1 or 2
+  int32_t K;                // images in the batch
+  IdxMap img0, img1;        // image index of batch n inside source 0 / 1
+  int32_t Ho, Wo;           // output extent
+  int32_t tiles_x, tiles_y; // 16 x 8 pixel patches
+  int32_t n_tiles_n;        // CoutPacked / block_n
+  int32_t block_n;          // 64, 128 or 256
+  int32_t cout;             // real output channels (RELU) or 4*hidden (LSTM)
+  int32_t epilogue;
+  const float* bias;        // packed order, [CoutPacked]
+  // RELU epilogue
+  __nv_bfloat16* out;       // [K][Ho][Wo][cout]
+  // LSTM epilogue
+  float* c_state;           // [slots][Hm][Wm][Ch] in place
+  float* h_f32;             // [slots][Hm][Wm][Ch]
+  __nv_bfloat16* h_bf16;    // [slots*2][Hm][Wm][Ch]
+  IdxMap c_idx, h_out_idx;  // slot, slot*2+half
+  int32_t hidden;
+  int32_t* status;          // device word: 0 ok, else a code describing a wait that ran out
+};
+cudaError_t launch_conv_tc(const ConvTcParams& p, int sm_count, cudaStream_t s);
+cudaError_t conv_tc_prepare();  // one-off function attribute set-up
+
+// ------------------------------------------------------------------- S4/S5 postprocess
+struct PostParams {
+  const float* h;       // fp32, image n at h + idx.v[n]*img_stride
+  int32_t channels_last;
+  int64_t img_stride;
+  IdxMap idx;
+  int32_t K, Hm, Wm, Ch, T;
+  const float* head_w;  // [T][Ch]
+  const float* head_b;
+  const float* conf_w;  // [T][Ch] or null
+  const float* conf_b;
+  int32_t conf_mode;
+  float zthr;
+  float* logits;        // [K][T][plane]
+  float* probs;
+  uint8_t* masks;
+  uint8_t* bits;        // optional [K][plane], bit t = mask of tool t
+  tt_result* results;   // device, [K]
+  void* scratch;
+};
+size_t post_scratch_bytes(int K, int hm, int wm, int ch, int T);
+cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s);
+cudaError_t post_prepare();
+
+// -------------------------------------------------------------------------- S6 overlay
+struct OverlayParams {
+  FramePtrs src;
+  int32_t K, src_w, src_h, src_pitch, T, Hm, Wm;
+  const uint8_t* masks;  // [K][T][plane] (used when bits == null)
+  const uint8_t* bits;   // [K][plane] packed
+  uint8_t palette[TT_MAX_TOOLS][3];
+  uint8_t* dst;          // [K][src_h][src_w][4]
+};
+cudaError_t launch_overlay(const OverlayParams& p, cudaStream_t s);
+
+// ------------------------------------------------------------------------ layout helpers
+// fp32 NCHW <-> internal layouts, used by state import/export and debug taps.
+cudaError_t launch_nhwc_to_nchw_f32(const float* src, float* dst, int C, int plane, cudaStream_t s);
+cudaError_t launch_nchw_to_nhwc_f32(const float* src, float* dst, int C, int plane, cudaStream_t s);
+cudaError_t launch_nhwc_bf16_to_nchw_f32(const __nv_bfloat16* src, float* dst, int C, int plane, cudaStream_t s);
+cudaError_t launch_nchw_f32_to_nhwc_bf16(const float* src, __nv_bfloat16* dst, int C, int plane, cudaStream_t s);
+
+}  // namespace tt
