@@ -255,6 +255,37 @@ tt_status tt_postprocess(const float* h_dev, int32_t channels_last, int32_t K, i
                          void* scratch_dev, void* cuda_stream);
 
 /*
+ * tt_postprocess_static — the same computation as tt_postprocess for callers that must not
+ * allocate device memory.  The paper has no counterpart for this call; it exists for users of
+ * this library that run where cudaMalloc is off limits: code inside a real-time frame loop
+ * that promised its host application a fixed memory footprint, plug-ins that are handed their
+ * buffers by a framework's own allocator, and callers that keep a whole device reserved by
+ * another pool.  Nothing is allocated or freed here, neither through CUDA nor through any
+ * library: the partial sums that tt_postprocess keeps in caller-provided scratch live in a
+ * fixed array of TT_POSTPROCESS_STATIC_SCRATCH_BYTES that is part of the library image (each
+ * GPU that loads the library holds that much memory until the process ends).  Inputs and
+ * outputs are still the caller's.
+ *
+ * Limits and rules:
+ *   - tt_postprocess_scratch_bytes(K, hm, wm, hidden, n_tools) must not exceed
+ *     TT_POSTPROCESS_STATIC_SCRATCH_BYTES, else TT_ERR_UNSUPPORTED is returned and nothing runs
+ *     (4 MiB covers 8 streams of a 160x90 grid with 256 hidden channels);
+ *   - the first call on a device looks up the array's device address (with that device
+ *     current); make that first call before starting any stream capture;
+ *   - all calls on a device share the one array.  It keeps whatever the previous call left;
+ *     every value that is read is written first within the same call, so nothing needs to be
+ *     cleared, but two calls whose kernels overlap on the GPU (different streams without an
+ *     ordering between them) race on it.  Serialise them.
+ * Everything else (arguments, layouts, outputs, errors) is as for tt_postprocess.
+ */
+#define TT_POSTPROCESS_STATIC_SCRATCH_BYTES (4u << 20)
+tt_status tt_postprocess_static(const float* h_dev, int32_t channels_last, int32_t K, int32_t hm, int32_t wm,
+                                int32_t hidden, int32_t n_tools, const float* head_w_dev, const float* head_b_dev,
+                                const float* conf_w_dev, const float* conf_b_dev, int32_t conf_mode, float threshold,
+                                float* logits_dev, float* probs_dev, uint8_t* masks_dev, tt_result* results_dev,
+                                void* cuda_stream);
+
+/*
  * tt_overlay — S6, the stand-in for the visualisation operator of Section II-B / III-A
  * (mask overlay on the frame).  src_dev as in tt_preprocess; masks_dev uint8
  * [K][n_tools][Hm][Wm]; palette: n_tools RGB triples (host); dst_dev uint8

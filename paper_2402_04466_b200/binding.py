@@ -28,8 +28,9 @@ EXPORTED_SYMBOLS = [
     "tt_abi_version", "tt_create", "tt_destroy", "tt_last_error", "tt_map_size", "tt_state_create",
     "tt_state_reset", "tt_state_export", "tt_state_import", "tt_submit_frames", "tt_sync", "tt_debug_tensor",
     "tt_set_profiling", "tt_get_stage_times", "tt_get_counters",
-    "tt_preprocess", "tt_postprocess_scratch_bytes", "tt_postprocess", "tt_overlay",
+    "tt_preprocess", "tt_postprocess_scratch_bytes", "tt_postprocess", "tt_postprocess_static", "tt_overlay",
 ]
+TT_POSTPROCESS_STATIC_SCRATCH_BYTES = 4 << 20
 STAGE_NAMES = ["h2d", "preprocess", "enc0", "enc1", "enc2", "enc3", "convlstm", "postprocess", "overlay"]
 
 
@@ -112,6 +113,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.tt_postprocess_scratch_bytes.argtypes = [i32, i32, i32, i32, i32]
     lib.tt_postprocess_scratch_bytes.restype = C.c_size_t
     lib.tt_postprocess.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp, vp]
+    lib.tt_postprocess_static.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp]
     lib.tt_overlay.argtypes = [vp, i32, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp]
     for name in EXPORTED_SYMBOLS:
         getattr(lib, name)  # AttributeError here means the library does not export what tt.h declares
@@ -375,6 +377,42 @@ def postprocess(h, channels_last: bool, head_w, head_b, conf_w=None, conf_b=None
     recs = [_result_to_dict(tt_result.from_buffer_copy(raw[k * C.sizeof(tt_result):(k + 1) * C.sizeof(tt_result)]), T)
             for k in range(K)]
     return {"logits": logits, "probs": probs, "masks": masks, "results": recs}
+
+
+def postprocess_static(h, channels_last: bool, head_w, head_b, conf_w=None, conf_b=None, conf_mode="mean_sigmoid",
+                       threshold=0.5, stream=None, out=None):
+    """tt_postprocess_static: like postprocess(), but the library call itself allocates nothing.
+
+    For callers that cannot allocate device memory while they run (a frame loop with a fixed
+    memory budget, a plug-in fed by its host's allocator).  The output tensors are the caller's:
+    pass them as `out` (dict with logits, probs, masks, results) to reuse buffers across calls;
+    when `out` is None this helper creates them with torch before calling into the library.
+    """
+    import torch
+    lib = load_library()
+    if channels_last:
+        K, hm, wm, ch = h.shape
+    else:
+        K, ch, hm, wm = h.shape
+    T = head_w.shape[0]
+    dev = h.device
+    if out is None:
+        out = {"logits": torch.empty((K, T, hm, wm), dtype=torch.float32, device=dev),
+               "probs": torch.empty((K, T, hm, wm), dtype=torch.float32, device=dev),
+               "masks": torch.empty((K, T, hm, wm), dtype=torch.uint8, device=dev),
+               "results_raw": torch.zeros((K, C.sizeof(tt_result)), dtype=torch.uint8, device=dev)}
+    mode = TT_CONF_GAP_LINEAR if conf_mode == "gap_linear" else TT_CONF_MEAN_SIGMOID
+    st = lib.tt_postprocess_static(h.data_ptr(), int(channels_last), K, hm, wm, ch, T, head_w.data_ptr(), head_b.data_ptr(),
+                                   conf_w.data_ptr() if conf_w is not None else None,
+                                   conf_b.data_ptr() if conf_b is not None else None, mode, threshold,
+                                   out["logits"].data_ptr(), out["probs"].data_ptr(), out["masks"].data_ptr(),
+                                   out["results_raw"].data_ptr(), _stream_ptr(stream))
+    _check(lib, st, None)
+    torch.cuda.synchronize()
+    raw = out["results_raw"].cpu().numpy().tobytes()
+    n = C.sizeof(tt_result)
+    out["results"] = [_result_to_dict(tt_result.from_buffer_copy(raw[k * n:(k + 1) * n]), T) for k in range(K)]
+    return out
 
 
 def overlay(src, src_w: int, src_h: int, src_pitch: int, masks, palette, stream=None):

@@ -7,6 +7,8 @@
 // as integers; sum p and per-channel sum h as floats) are written to scratch.
 // Pass 2 (post_finalize_kernel): one block per stream adds the partials in a fixed order
 // (bitwise reproducible, no float atomics) and forms confidence and centroid.
+#include <mutex>
+
 #include "tt_internal.h"
 
 namespace tt {
@@ -215,6 +217,10 @@ __global__ void __launch_bounds__(POST_THREADS) post_finalize_kernel(const PostP
   }
 }
 
+// Scratch of the entry point that allocates nothing: one fixed array inside the library image.
+// Every device that loads the library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_static_post_scratch[TT_POSTPROCESS_STATIC_SCRATCH_BYTES];
+
 size_t post_smem_bytes(int ch) {
   return (size_t)(PIX * (ch + ROW_PAD) + TT_MAX_TOOLS * ch + 8 * TT_MAX_TOOLS) * sizeof(float) +
          (size_t)8 * TT_MAX_TOOLS * 3 * sizeof(int);
@@ -223,6 +229,27 @@ size_t post_smem_bytes(int ch) {
 }  // namespace
 
 size_t post_scratch_bytes(int K, int hm, int wm, int ch, int T) { return scratch_layout(K, hm * wm, ch, T).total; }
+
+// In host code the array's name is only a handle; the device address has to be asked for,
+// once per device, with that device current.
+cudaError_t post_static_scratch(void** ptr) {
+  constexpr int MAX_DEV = 64;
+  static void* addr[MAX_DEV] = {};
+  static std::mutex mu;
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= MAX_DEV) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lk(mu);
+  if (!addr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_post_scratch);
+    if (e != cudaSuccess) return e;
+    addr[dev] = p;
+  }
+  *ptr = addr[dev];
+  return cudaSuccess;
+}
 
 cudaError_t post_prepare() {
   return cudaFuncSetAttribute(post_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)post_smem_bytes(512));

@@ -936,6 +936,44 @@ tt_status tt_postprocess(const float* h_dev, int32_t channels_last, int32_t K, i
   return TT_OK;
 }
 
+// Variant of tt_postprocess for callers that cannot allocate: same kernels, scratch taken from
+// the array built into the library.  No allocation or free happens on this path.
+tt_status tt_postprocess_static(const float* h_dev, int32_t channels_last, int32_t K, int32_t hm, int32_t wm,
+                                int32_t hidden, int32_t n_tools, const float* head_w_dev, const float* head_b_dev,
+                                const float* conf_w_dev, const float* conf_b_dev, int32_t conf_mode, float threshold,
+                                float* logits_dev, float* probs_dev, uint8_t* masks_dev, tt_result* results_dev,
+                                void* cuda_stream) {
+  if (!h_dev || !head_w_dev || !head_b_dev || !logits_dev || !probs_dev || !masks_dev || !results_dev || K < 1 ||
+      K > TT_MAX_STREAMS || hm < 1 || wm < 1 || n_tools < 1 || n_tools > TT_MAX_TOOLS ||
+      !(threshold > 0.f && threshold < 1.f) || (conf_mode != TT_CONF_MEAN_SIGMOID && conf_mode != TT_CONF_GAP_LINEAR) ||
+      (conf_mode == TT_CONF_GAP_LINEAR && (!conf_w_dev || !conf_b_dev)))
+    return fail(nullptr, TT_ERR_INVALID_ARG, "tt_postprocess_static: bad argument");
+  if (hidden < 4 || hidden > 512 || hidden % 4)
+    return fail(nullptr, TT_ERR_UNSUPPORTED, "tt_postprocess_static: hidden must be a multiple of 4 in [4, 512]");
+  const size_t need = post_scratch_bytes(K, hm, wm, hidden, n_tools);
+  if (need > (size_t)TT_POSTPROCESS_STATIC_SCRATCH_BYTES)
+    return fail(nullptr, TT_ERR_UNSUPPORTED,
+                "tt_postprocess_static: this problem needs %zu bytes of scratch, the built-in array holds %u; "
+                "use tt_postprocess with caller-provided scratch",
+                need, (unsigned)TT_POSTPROCESS_STATIC_SCRATCH_BYTES);
+  void* scratch = nullptr;
+  cudaError_t e = post_static_scratch(&scratch);
+  if (e != cudaSuccess) return fail(nullptr, TT_ERR_CUDA, "tt_postprocess_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+  e = post_prepare();
+  if (e != cudaSuccess) return fail(nullptr, TT_ERR_CUDA, "tt_postprocess_static: %s", cudaGetErrorString(e));
+  PostParams p{};
+  p.h = h_dev; p.channels_last = channels_last; p.img_stride = (int64_t)hidden * hm * wm;
+  for (int n = 0; n < TT_MAX_STREAMS; ++n) p.idx.v[n] = n;
+  p.K = K; p.Hm = hm; p.Wm = wm; p.Ch = hidden; p.T = n_tools;
+  p.head_w = head_w_dev; p.head_b = head_b_dev; p.conf_w = conf_w_dev; p.conf_b = conf_b_dev; p.conf_mode = conf_mode;
+  p.zthr = (float)std::log((double)threshold / (1.0 - (double)threshold));
+  p.logits = logits_dev; p.probs = probs_dev; p.masks = masks_dev; p.bits = nullptr; p.results = results_dev;
+  p.scratch = scratch;
+  e = launch_postprocess(p, reinterpret_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return fail(nullptr, TT_ERR_CUDA, "tt_postprocess_static: %s", cudaGetErrorString(e));
+  return TT_OK;
+}
+
 tt_status tt_overlay(const uint8_t* src_dev, int32_t K, int64_t src_frame_stride, int32_t src_w, int32_t src_h,
                      int32_t src_pitch, const uint8_t* masks_dev, int32_t n_tools, int32_t hm, int32_t wm,
                      const uint8_t* palette_host, uint8_t* dst_dev, void* cuda_stream) {

@@ -119,6 +119,7 @@ struct PostParams {
 size_t post_scratch_bytes(int K, int hm, int wm, int ch, int T);
 cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s);
 cudaError_t post_prepare();
+cudaError_t post_static_scratch(void** ptr);  // device address of the library's built-in scratch array
 
 // -------------------------------------------------------------------------- S6 overlay
 struct OverlayParams {
