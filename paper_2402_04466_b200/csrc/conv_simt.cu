@@ -37,7 +37,7 @@ __device__ __forceinline__ void store_bf16_vec(__nv_bfloat16* dst, const float* 
 __device__ __forceinline__ float sigmoid_acc(float z) { return 1.0f / (1.0f + expf(-z)); }
 
 template <int STRIDE, int EPI, int OCB>
-__global__ void __launch_bounds__(TW* TH) conv3x3_simt_kernel(const ConvSimtParams p) {
+__global__ void __launch_bounds__(TW* TH) conv3x3_simt_kernel(const __grid_constant__ ConvSimtParams p) {
   constexpr int IN_W = TW * STRIDE + 2;
   constexpr int IN_H = TH * STRIDE + 2;
   constexpr int IN_WP = IN_W + 1;  // pad against bank conflicts

@@ -13,8 +13,9 @@
 // columns), each an ordinary tiled tensor map with doubled strides, so every tap is again
 // a dense box.
 //
-// Warp roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM allocation and
-// MMA issue (one lane), warps 2..5 = epilogue (TMEM lane quarter = warp index mod 4).
+// Warp roles (320 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM allocation and
+// MMA issue (one lane), warps 2..9 = epilogue (TMEM lane quarter = warp index mod 4, two warps
+// per quarter, each taking half of the tile's columns).
 // Every mbarrier wait is bounded: when a wait runs out the kernel records a status code,
 // raises a block-wide abort flag, lets copies in flight land, frees its TMEM and returns.
 #include "tt_internal.h"
@@ -25,7 +26,8 @@ namespace {
 constexpr int BLOCK_M = 128;
 constexpr int PATCH_W = 16, PATCH_H = 8;
 constexpr int UMMA_K = 16;
-constexpr int TC_THREADS = 192;
+constexpr int EPI_WARPS = 8;                       // two per TMEM lane quarter, each takes half of the columns
+constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s per wait
 
 template <int BLOCK_N, int SLAB_C>
@@ -150,8 +152,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-__device__ __forceinline__ float fast_sigmoid(float z) { return __frcp_rn(1.0f + __expf(-z)); }
-__device__ __forceinline__ float fast_tanh(float z) { return 1.0f - 2.0f * __frcp_rn(1.0f + __expf(2.0f * z)); }
+// One special-function instruction each: tanh.approx (relative error about 2^-11, far inside
+// the bf16 path's tolerance) and sigmoid(z) = 0.5 + 0.5 * tanh(z / 2).
+__device__ __forceinline__ float fast_tanh(float z) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(z));
+  return y;
+}
+__device__ __forceinline__ float fast_sigmoid(float z) { return fmaf(0.5f, fast_tanh(0.5f * z), 0.5f); }
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
@@ -186,7 +194,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(tfull_bar + a), 1);
-      mbar_init(smem_u32(tempty_bar + a), 4);
+      mbar_init(smem_u32(tempty_bar + a), EPI_WARPS);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -280,7 +288,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     }
   } else if (warp >= 2) {
     // ---------------------------------------------------------------------- epilogue
+    constexpr int HALF_N = BLOCK_N / 2;           // columns handled by this warp
+    constexpr int CHUNKS = HALF_N / 32;
     const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
+    const int half = (warp - 2) >> 2;             // which half of the tile's columns
     const int row = quarter * 32 + lane;          // row of the 128-row tile = pixel of the patch
     const int py = row / PATCH_W, px = row % PATCH_W;
     uint32_t acc_phase = 0;
@@ -292,16 +303,37 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
       const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
       const int x = tx * PATCH_W + px, y = ty * PATCH_H + py;
       const bool valid = x < p.Wo && y < p.Ho;
+      const size_t pix = (size_t)y * p.Wo + x;
+      const int col0 = nt * BLOCK_N + half * HALF_N;  // first packed output column of this warp
+
+      // The old cell state of this thread's pixel is fetched before the accumulator is
+      // waited for, so its latency hides under the tile's main loop.
+      float c_old[EPI == TC_EPI_LSTM ? CHUNKS * 8 : 1];
+      size_t so = 0, ho = 0;
+      if (EPI == TC_EPI_LSTM) {
+        so = ((size_t)p.c_idx.v[img] * p.Ho * p.Wo + pix) * p.hidden + (col0 >> 2);
+        ho = ((size_t)p.h_out_idx.v[img] * p.Ho * p.Wo + pix) * p.hidden + (col0 >> 2);
+#pragma unroll
+        for (int ck = 0; ck < CHUNKS; ++ck) {
+          float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+          if (valid && (col0 >> 2) + ck * 8 < p.hidden) {
+            lo = *reinterpret_cast<const float4*>(p.c_state + so + ck * 8);
+            hi = *reinterpret_cast<const float4*>(p.c_state + so + ck * 8 + 4);
+          }
+          c_old[ck * 8 + 0] = lo.x; c_old[ck * 8 + 1] = lo.y; c_old[ck * 8 + 2] = lo.z; c_old[ck * 8 + 3] = lo.w;
+          c_old[ck * 8 + 4] = hi.x; c_old[ck * 8 + 5] = hi.y; c_old[ck * 8 + 6] = hi.z; c_old[ck * 8 + 7] = hi.w;
+        }
+      }
+
       ok = mbar_wait(smem_u32(tfull_bar + acc), acc_phase, abort_flag, p.status, 0x400 + acc);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
-      const size_t pix = (size_t)y * p.Wo + x;
-#pragma unroll 1
-      for (int ch0 = 0; ch0 < BLOCK_N; ch0 += 32) {
+      const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N + half * HALF_N);
+#pragma unroll
+      for (int ck = 0; ck < CHUNKS; ++ck) {
         uint32_t v[32];
-        tmem_ld32(t_addr + (uint32_t)ch0, v);
-        const int n0 = nt * BLOCK_N + ch0;        // first packed output column of this chunk
+        tmem_ld32(t_addr + (uint32_t)(ck * 32), v);
+        const int n0 = col0 + ck * 32;            // first packed output column of this chunk
         if (EPI == TC_EPI_RELU_BF16) {
           if (valid && n0 < p.cout) {
             const float4* b4 = reinterpret_cast<const float4*>(p.bias + n0);
@@ -319,16 +351,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
           }
         } else {
           // packed column = 4*jj + gate (i, f, g, o); 8 hidden units per 32-column chunk
-          const int j0 = n0 >> 2;
-          if (valid && j0 < p.hidden) {
+          if (valid && (n0 >> 2) < p.hidden) {
             const float4* b4 = reinterpret_cast<const float4*>(p.bias + n0);
-            const size_t so = ((size_t)p.c_idx.v[img] * p.Ho * p.Wo + pix) * p.hidden + j0;
-            const size_t ho = ((size_t)p.h_out_idx.v[img] * p.Ho * p.Wo + pix) * p.hidden + j0;
-            float* c_ptr = p.c_state + so;
-            float* h_ptr = p.h_f32 + so;
-            const float4 c_lo = *reinterpret_cast<const float4*>(c_ptr);
-            const float4 c_hi = *reinterpret_cast<const float4*>(c_ptr + 4);
-            const float c_old[8] = {c_lo.x, c_lo.y, c_lo.z, c_lo.w, c_hi.x, c_hi.y, c_hi.z, c_hi.w};
             float c_new[8], h_new[8];
 #pragma unroll
             for (int jj = 0; jj < 8; ++jj) {
@@ -337,9 +361,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
               const float gf = __uint_as_float(v[4 * jj + 1]) + b.y;
               const float gg = __uint_as_float(v[4 * jj + 2]) + b.z;
               const float go = __uint_as_float(v[4 * jj + 3]) + b.w;
-              c_new[jj] = fast_sigmoid(gf) * c_old[jj] + fast_sigmoid(gi) * fast_tanh(gg);
+              c_new[jj] = fast_sigmoid(gf) * c_old[ck * 8 + jj] + fast_sigmoid(gi) * fast_tanh(gg);
               h_new[jj] = fast_sigmoid(go) * fast_tanh(c_new[jj]);
             }
+            float* c_ptr = p.c_state + so + ck * 8;
+            float* h_ptr = p.h_f32 + so + ck * 8;
             *reinterpret_cast<float4*>(c_ptr) = make_float4(c_new[0], c_new[1], c_new[2], c_new[3]);
             *reinterpret_cast<float4*>(c_ptr + 4) = make_float4(c_new[4], c_new[5], c_new[6], c_new[7]);
             *reinterpret_cast<float4*>(h_ptr) = make_float4(h_new[0], h_new[1], h_new[2], h_new[3]);
@@ -349,7 +375,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
             hb.y = pack_bf16(h_new[2], h_new[3]);
             hb.z = pack_bf16(h_new[4], h_new[5]);
             hb.w = pack_bf16(h_new[6], h_new[7]);
-            *reinterpret_cast<uint4*>(p.h_bf16 + ho) = hb;
+            *reinterpret_cast<uint4*>(p.h_bf16 + ho + ck * 8) = hb;
           }
         }
       }

@@ -31,7 +31,7 @@ __device__ __forceinline__ uint32_t blend_px(int r, int g, int b, uint32_t bits,
 }
 
 template <bool PACKED, bool FLAT>
-__global__ void __launch_bounds__(256) overlay_kernel(const OverlayParams p) {
+__global__ void __launch_bounds__(256) overlay_kernel(const __grid_constant__ OverlayParams p) {
   const int n = blockIdx.y;
   const uint8_t* __restrict__ src = p.src.p[n];
   const long long npx = (long long)p.src_w * p.src_h;

@@ -36,7 +36,7 @@ __host__ __device__ inline ScratchLayout scratch_layout(int K, int plane, int ch
 
 __device__ __forceinline__ float sigmoid_acc(float z) { return 1.0f / (1.0f + expf(-z)); }
 
-__global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const PostParams p) {
+__global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const __grid_constant__ PostParams p) {
   extern __shared__ __align__(16) float s_mem[];
   const int Ch = p.Ch, T = p.T;
   const int row = Ch + ROW_PAD;
@@ -161,6 +161,7 @@ __global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const PostParam
     part_i[tid * 4 + 0] = cnt;
     part_i[tid * 4 + 1] = sx;
     part_i[tid * 4 + 2] = sy;
+    part_i[tid * 4 + 3] = 0;
     part_p[tid] = sp;
   }
   if (p.conf_mode == TT_CONF_GAP_LINEAR) {
@@ -172,48 +173,71 @@ __global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const PostParam
   }
 }
 
-__global__ void __launch_bounds__(POST_THREADS) post_finalize_kernel(const PostParams p) {
+// One block of 1024 threads per stream.  Pooled hidden state: the tile blocks are split into
+// G = 1024 / Ch interleaved groups, thread (g, c) adds channel c over group g's blocks in
+// order, and the G group sums are added in order.  Tool statistics: warp t reduces the partials
+// of tool t (lanes stride over the tile blocks, then a fixed shuffle tree).  The order of the
+// additions never depends on timing, so results are bitwise reproducible.
+constexpr int FIN_THREADS = 1024;
+
+__global__ void __launch_bounds__(FIN_THREADS) post_finalize_kernel(const __grid_constant__ PostParams p) {
+  __shared__ float s_part[FIN_THREADS];
   __shared__ float s_gap[512];
-  const int n = blockIdx.x, tid = threadIdx.x;
+  const int n = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int plane = p.Hm * p.Wm, Ch = p.Ch, T = p.T;
   const int nb = post_blocks_per_img(plane);
   const ScratchLayout sl = scratch_layout(p.K, plane, Ch, T);
   const uint8_t* scr = reinterpret_cast<const uint8_t*>(p.scratch);
-  const int32_t* part_i = reinterpret_cast<const int32_t*>(scr + sl.off_int) + (size_t)n * nb * TT_MAX_TOOLS * 4;
+  const int4* part_i = reinterpret_cast<const int4*>(scr + sl.off_int) + (size_t)n * nb * TT_MAX_TOOLS;
   const float* part_p = reinterpret_cast<const float*>(scr + sl.off_p) + (size_t)n * nb * TT_MAX_TOOLS;
   const float* part_h = reinterpret_cast<const float*>(scr + sl.off_h) + (size_t)n * nb * Ch;
   const float inv_plane = 1.0f / (float)plane;
 
   if (p.conf_mode == TT_CONF_GAP_LINEAR) {
-    for (int c = tid; c < Ch; c += POST_THREADS) {
-      float s = 0.0f;
-      for (int b = 0; b < nb; ++b) s += part_h[(size_t)b * Ch + c];
-      s_gap[c] = s * inv_plane;
+    const int G = FIN_THREADS / Ch;          // Ch <= 512, so G >= 2
+    const int g = tid / Ch, c = tid - g * Ch;
+    float s = 0.0f;
+    if (g < G) {
+#pragma unroll 8
+      for (int b = g; b < nb; b += G) s += part_h[(size_t)b * Ch + c];
+    }
+    s_part[tid] = s;
+    __syncthreads();
+    if (tid < Ch) {
+      float a = 0.0f;
+      for (int k = 0; k < G; ++k) a += s_part[k * Ch + tid];
+      s_gap[tid] = a * inv_plane;
     }
   }
   __syncthreads();
-  if (tid < T) {
+  if (warp < T) {
+    const int t = warp;
     long long cnt = 0, sx = 0, sy = 0;
     float sp = 0.0f;
-    for (int b = 0; b < nb; ++b) {
-      cnt += part_i[((size_t)b * TT_MAX_TOOLS + tid) * 4 + 0];
-      sx += part_i[((size_t)b * TT_MAX_TOOLS + tid) * 4 + 1];
-      sy += part_i[((size_t)b * TT_MAX_TOOLS + tid) * 4 + 2];
-      sp += part_p[(size_t)b * TT_MAX_TOOLS + tid];
+    for (int b = lane; b < nb; b += 32) {
+      const int4 v = part_i[(size_t)b * TT_MAX_TOOLS + t];
+      cnt += v.x; sx += v.y; sy += v.z;
+      sp += part_p[(size_t)b * TT_MAX_TOOLS + t];
     }
-    float conf;
-    if (p.conf_mode == TT_CONF_GAP_LINEAR) {
-      float a = __ldg(p.conf_b + tid);
-      for (int c = 0; c < Ch; ++c) a = fmaf(__ldg(p.conf_w + tid * Ch + c), s_gap[c], a);
-      conf = sigmoid_acc(a);
-    } else {
-      conf = sp * inv_plane;
+    float a = 0.0f;
+    if (p.conf_mode == TT_CONF_GAP_LINEAR)
+      for (int c = lane; c < Ch; c += 32) a = fmaf(__ldg(p.conf_w + t * Ch + c), s_gap[c], a);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+      sx += __shfl_xor_sync(0xffffffffu, sx, d);
+      sy += __shfl_xor_sync(0xffffffffu, sy, d);
+      sp += __shfl_xor_sync(0xffffffffu, sp, d);
+      a += __shfl_xor_sync(0xffffffffu, a, d);
     }
-    tt_result* r = p.results + n;
-    r->conf[tid] = conf;
-    r->count[tid] = (int32_t)cnt;
-    r->cx[tid] = cnt ? (float)((double)sx / (double)cnt) : -1.0f;
-    r->cy[tid] = cnt ? (float)((double)sy / (double)cnt) : -1.0f;
+    if (lane == 0) {
+      const float conf = p.conf_mode == TT_CONF_GAP_LINEAR ? sigmoid_acc(a + __ldg(p.conf_b + t)) : sp * inv_plane;
+      tt_result* r = p.results + n;
+      r->conf[t] = conf;
+      r->count[t] = (int32_t)cnt;
+      r->cx[t] = cnt ? (float)((double)sx / (double)cnt) : -1.0f;
+      r->cy[t] = cnt ? (float)((double)sy / (double)cnt) : -1.0f;
+    }
   }
 }
 
@@ -261,7 +285,7 @@ cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s) {
   post_tile_kernel<<<p.K * nb, POST_THREADS, post_smem_bytes(p.Ch), s>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  post_finalize_kernel<<<p.K, POST_THREADS, 0, s>>>(p);
+  post_finalize_kernel<<<p.K, FIN_THREADS, 0, s>>>(p);
   return cudaGetLastError();
 }
 

@@ -56,6 +56,19 @@ struct ConvSimtParams {
 };
 cudaError_t launch_conv_simt(const ConvSimtParams& p, cudaStream_t s);
 
+// --------------------------------------- S2 first encoder layer of the bf16 path (Cin = 3)
+// Passed by value: the weights sit in the kernel parameter block (constant bank).
+constexpr int CONV_FIRST_MAX_COUT = 64;
+struct ConvFirstParams {
+  const float* in;       // [K][3][H][W] fp32
+  __nv_bfloat16* out;    // [K][Ho][Wo][cout] bf16
+  int32_t H, W, Ho, Wo, stride, K, cout;
+  float w[27 * CONV_FIRST_MAX_COUT];  // [(c*3+ky)*3+kx][cout]
+  float b[CONV_FIRST_MAX_COUT];
+};
+bool conv_first_supported(int cout);
+cudaError_t launch_conv_first(const ConvFirstParams& p, cudaStream_t s);
+
 // ------------------------------------------------- S2/S3 tcgen05 implicit-GEMM conv (bf16)
 // One launch description; tensor maps live in device-visible constant storage owned by the
 // caller (passed by value as __grid_constant__ kernel parameters).
