@@ -35,8 +35,8 @@ class OraclePipeline:
     """One stream: weights + (h, c).  `wl` is any object with the Workload attributes.
 
     mirror_bf16=True rounds to bf16 exactly those activations that a bf16 tensor-core path
-    must round before a contraction (every encoder output and the copy of h fed back into
-    the ConvLSTM convolution); state, heads and everything observable stay fp32.
+    must round before a contraction (the network input of the first layer, every encoder
+    output and the copy of h fed back into the ConvLSTM convolution); state, heads and everything observable stay fp32.
     """
 
     def __init__(self, wl, weights: Dict[str, np.ndarray], mirror_bf16: bool = False):
@@ -58,7 +58,7 @@ class OraclePipeline:
     def step(self, frame: np.ndarray, want_overlay: Optional[bool] = None) -> FrameOutput:
         wl, w = self.wl, self.w
         pre = S.preprocess(frame, wl.net_w, wl.net_h, wl.norm_div, wl.norm_mean, wl.norm_std)
-        a = pre
+        a = S.round_bf16(pre) if self.mirror else pre     # the first contraction also takes bf16 operands
         enc = []
         for l, s in enumerate(wl.enc_stride):
             a = S.conv3x3(a, w[f"enc_w{l}"], w[f"enc_b{l}"], stride=s, relu=True)

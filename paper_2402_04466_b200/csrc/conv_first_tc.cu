@@ -1,0 +1,207 @@
+// First encoder layer of the bf16 path on the tensor cores: 3 input channels (planar fp32 from
+// preprocess) -> COUT channels, 3x3, pad 1, stride 1 or 2, bias, ReLU, output bf16 channels-last.
+//
+// K = 27 (padded to 32) makes the arithmetic free on tcgen05; the layer is then bound by HBM
+// (read the fp32 input once, write the bf16 output once).  The A operand cannot come from TMA
+// (planar fp32 source, 3 channels), so four producer warps build it: each thread gathers the
+// 27 taps of one output pixel, rounds them to bf16 and writes one 64-byte row of the
+// [128 pixels][32] operand tile in the no-swizzle K-major core-matrix layout (8 rows x 16 bytes
+// contiguous; neighbouring core matrices 128 bytes apart along K, 512 bytes apart along M).
+// One warp issues two M128 x COUT x K16 MMAs per tile; four warps run the bias + ReLU epilogue
+// from TMEM.  The operand ring has 4 stages and the accumulator 2 buffers, so gather, MMA and
+// epilogue of different tiles overlap.  All waits are bounded (see tc_ptx.cuh).
+#include "tt_internal.h"
+#include "tc_ptx.cuh"
+
+namespace tt {
+namespace {
+
+using namespace tc;
+
+constexpr int F_STAGES = 4;
+constexpr int F_A_BYTES = 128 * 64;                 // 128 rows x 32 bf16
+constexpr int F_THREADS = 288;                      // warps 0-3 gather, 4 MMA, 5-8 epilogue
+constexpr int F_TMEM_COLS = 128;                    // two accumulator buffers of up to 64 columns
+
+template <int COUT>
+__global__ void __launch_bounds__(F_THREADS) conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
+  __shared__ __align__(1024) uint8_t s_a[F_STAGES * F_A_BYTES];
+  __shared__ __align__(1024) uint8_t s_b[COUT * 64];
+  __shared__ __align__(8) uint64_t s_bar[2 * F_STAGES + 4];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+  uint64_t* a_full = s_bar;                 // [F_STAGES] 128 gather threads arrive
+  uint64_t* a_empty = s_bar + F_STAGES;     // [F_STAGES] MMA commit
+  uint64_t* t_full = s_bar + 2 * F_STAGES;  // [2] MMA commit
+  uint64_t* t_empty = t_full + 2;           // [2] 4 epilogue warps arrive
+  volatile int* abort_flag = &s_abort;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < F_STAGES; ++s) {
+      mbar_init(smem_u32(a_full + s), 128);
+      mbar_init(smem_u32(a_empty + s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(t_full + a), 1);
+      mbar_init(smem_u32(t_empty + a), 4);
+    }
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // weights: already packed in the operand layout, COUT * 64 bytes
+  for (int i = threadIdx.x; i < COUT * 4; i += F_THREADS)
+    reinterpret_cast<uint4*>(s_b)[i] = __ldg(reinterpret_cast<const uint4*>(p.w_packed) + i);
+  fence_proxy_async_smem();
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)),
+                 "r"((uint32_t)F_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = s_tmem;
+
+  const int tiles_per_img = p.tiles_x * p.tiles_y;
+  const int total_tiles = p.K * tiles_per_img;
+  const size_t in_plane = (size_t)p.H * p.W;
+
+  if (warp < 4) {
+    // ------------------------------------------------------------------ gather producers
+    const int row = warp * 32 + lane;
+    const int py = row >> 4, px = row & 15;
+    uint8_t* my_row = s_a + (row >> 3) * 512 + (row & 7) * 16;   // + kc * 128 per 16-byte chunk
+    uint32_t stage = 0, phase = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, img = tile / tiles_per_img;
+      const int xo = tx * 16 + px, yo = ty * 8 + py;
+      const bool valid = xo < p.Wo && yo < p.Ho;
+      const float* src = p.in + (size_t)img * 3 * in_plane;
+      const int x0 = xo * p.stride - 1, y0 = yo * p.stride - 1;
+      float v[27];
+#pragma unroll
+      for (int c = 0; c < 3; ++c)
+#pragma unroll
+        for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+          for (int kx = 0; kx < 3; ++kx) {
+            const int yi = y0 + ky, xi = x0 + kx;
+            const bool ok = valid && yi >= 0 && yi < p.H && xi >= 0 && xi < p.W;
+            v[(c * 3 + ky) * 3 + kx] = ok ? __ldg(src + (size_t)c * in_plane + (size_t)yi * p.W + xi) : 0.0f;
+          }
+      if (!mbar_wait(smem_u32(a_empty + stage), phase ^ 1u, abort_flag, p.status, 0x500 + (int)stage)) break;
+      uint8_t* dst = my_row + stage * F_A_BYTES;
+      uint4 u;
+      u.x = pack_bf16(v[0], v[1]);   u.y = pack_bf16(v[2], v[3]);   u.z = pack_bf16(v[4], v[5]);   u.w = pack_bf16(v[6], v[7]);
+      *reinterpret_cast<uint4*>(dst) = u;
+      u.x = pack_bf16(v[8], v[9]);   u.y = pack_bf16(v[10], v[11]); u.z = pack_bf16(v[12], v[13]); u.w = pack_bf16(v[14], v[15]);
+      *reinterpret_cast<uint4*>(dst + 128) = u;
+      u.x = pack_bf16(v[16], v[17]); u.y = pack_bf16(v[18], v[19]); u.z = pack_bf16(v[20], v[21]); u.w = pack_bf16(v[22], v[23]);
+      *reinterpret_cast<uint4*>(dst + 256) = u;
+      u.x = pack_bf16(v[24], v[25]); u.y = pack_bf16(v[26], 0.f);   u.z = 0u;                      u.w = 0u;
+      *reinterpret_cast<uint4*>(dst + 384) = u;
+      fence_proxy_async_smem();
+      mbar_arrive(smem_u32(a_full + stage));
+      if (++stage == F_STAGES) { stage = 0; phase ^= 1u; }
+    }
+  } else if (warp == 4) {
+    // ------------------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t IDESC = make_idesc(128, COUT);
+      uint32_t stage = 0, phase = 0, acc_phase = 0;
+      int acc = 0;
+      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        if (!mbar_wait(smem_u32(t_empty + acc), acc_phase ^ 1u, abort_flag, p.status, 0x600 + acc)) break;
+        if (!mbar_wait(smem_u32(a_full + stage), phase, abort_flag, p.status, 0x700 + (int)stage)) break;
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(s_a + stage * F_A_BYTES), b_addr = smem_u32(s_b);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 64);
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          // K step k covers the 16-byte chunks 2k and 2k+1 of every row: 256 bytes further on
+          const uint64_t a_desc = make_smem_desc_lbo(a_addr + k * 256, 128, 512, 0);
+          const uint64_t b_desc = make_smem_desc_lbo(b_addr + k * 256, 128, 512, 0);
+          umma_bf16(d_tmem, a_desc, b_desc, IDESC, k);
+        }
+        umma_commit(smem_u32(a_empty + stage));
+        umma_commit(smem_u32(t_full + acc));
+        if (++stage == F_STAGES) { stage = 0; phase ^= 1u; }
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // --------------------------------------------------------------------------- epilogue
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int py = row >> 4, px = row & 15;
+    uint32_t acc_phase = 0;
+    int acc = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, img = tile / tiles_per_img;
+      const int xo = tx * 16 + px, yo = ty * 8 + py;
+      const bool valid = xo < p.Wo && yo < p.Ho;
+      if (!mbar_wait(smem_u32(t_full + acc), acc_phase, abort_flag, p.status, 0x800 + acc)) break;
+      tc_fence_after();
+      const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 64);
+      __nv_bfloat16* dst = p.out + (((size_t)img * p.Ho + yo) * p.Wo + xo) * COUT;
+#pragma unroll
+      for (int ck = 0; ck < COUT / 32; ++ck) {
+        uint32_t v[32];
+        tmem_ld32(t_addr + (uint32_t)(ck * 32), v);
+        if (valid) {
+          const float4* b4 = reinterpret_cast<const float4*>(p.bias + ck * 32);
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            const float4 ba = __ldg(b4 + i / 4), bb = __ldg(b4 + i / 4 + 1);
+            uint4 u;
+            u.x = pack_bf16(fmaxf(__uint_as_float(v[i + 0]) + ba.x, 0.f), fmaxf(__uint_as_float(v[i + 1]) + ba.y, 0.f));
+            u.y = pack_bf16(fmaxf(__uint_as_float(v[i + 2]) + ba.z, 0.f), fmaxf(__uint_as_float(v[i + 3]) + ba.w, 0.f));
+            u.z = pack_bf16(fmaxf(__uint_as_float(v[i + 4]) + bb.x, 0.f), fmaxf(__uint_as_float(v[i + 5]) + bb.y, 0.f));
+            u.w = pack_bf16(fmaxf(__uint_as_float(v[i + 6]) + bb.z, 0.f), fmaxf(__uint_as_float(v[i + 7]) + bb.w, 0.f));
+            *reinterpret_cast<uint4*>(dst + ck * 32 + i) = u;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(t_empty + acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  __syncwarp();
+  if (*abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(16000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)F_TMEM_COLS)
+                 : "memory");
+  }
+}
+
+}  // namespace
+
+bool conv_first_tc_supported(int cout) { return cout == 32 || cout == 64; }
+
+// [cout][27] bf16 bit patterns (row-major, k = c*9 + ky*3 + kx) -> operand layout, cout*32 values
+void conv_first_tc_pack(const uint16_t* w_bf16, int cout, uint16_t* packed) {
+  for (int n = 0; n < cout; ++n)
+    for (int k = 0; k < 32; ++k)
+      packed[((n >> 3) * 4 + (k >> 3)) * 64 + (n & 7) * 8 + (k & 7)] = k < 27 ? w_bf16[n * 27 + k] : (uint16_t)0;
+}
+
+cudaError_t launch_conv_first_tc(const ConvFirstTcParams& p, int sm_count, cudaStream_t s) {
+  const int total = p.K * p.tiles_x * p.tiles_y;
+  const int grid = total < 3 * sm_count ? total : 3 * sm_count;
+  if (p.cout == 32) conv_first_tc_kernel<32><<<grid, F_THREADS, 0, s>>>(p);
+  else if (p.cout == 64) conv_first_tc_kernel<64><<<grid, F_THREADS, 0, s>>>(p);
+  else return cudaErrorInvalidValue;
+  return cudaGetLastError();
+}
+
+}  // namespace tt

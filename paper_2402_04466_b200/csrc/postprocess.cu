@@ -173,6 +173,160 @@ __global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const __grid_co
   }
 }
 
+// Channels-last fast path (hidden a multiple of 128): no shared-memory staging of the hidden
+// state.  A warp takes 8 of the block's 64 pixels, 4 at a time.  Lane l owns channels
+// [128*k + 4*l, +4) of every 128-channel chunk k, so each load instruction of a warp reads 512
+// contiguous bytes.  The lane's partial dot products for (4 pixels x 8 tool slots) = 32 values
+// are summed across the warp by a transposing butterfly (31 shuffles for all 32 values, fixed
+// order), after which lane i holds the logit of pixel i/8, tool i%8.  The pooled hidden state
+// accumulates in registers on the way.
+template <int NCHUNK>
+__global__ void __launch_bounds__(POST_THREADS) post_direct_kernel(const __grid_constant__ PostParams p) {
+  constexpr int CH = NCHUNK * 128;
+  __shared__ __align__(16) float s_w[TT_MAX_TOOLS * CH];
+  __shared__ __align__(16) float s_gapw[8][CH];
+  __shared__ float s_red_f[8 * TT_MAX_TOOLS];
+  __shared__ int s_red_i[8 * TT_MAX_TOOLS * 3];
+
+  const int T = p.T;
+  const int plane = p.Hm * p.Wm;
+  const int nb = post_blocks_per_img(plane);
+  const int n = blockIdx.x / nb, blk = blockIdx.x % nb;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const float* h_img = p.h + (size_t)p.idx.v[n] * p.img_stride;
+
+  for (int i = tid; i < TT_MAX_TOOLS * CH; i += POST_THREADS) s_w[i] = i < T * CH ? __ldg(p.head_w + i) : 0.0f;
+  __syncthreads();
+
+  const int slot = lane >> 3, t = lane & 7;       // after the butterfly this lane owns (pixel slot, tool)
+  const float bias = t < T ? __ldg(p.head_b + t) : 0.0f;
+  float gap[NCHUNK * 4];
+#pragma unroll
+  for (int i = 0; i < NCHUNK * 4; ++i) gap[i] = 0.0f;
+  int cnt = 0, sx = 0, sy = 0;
+  float sp = 0.0f;
+
+#pragma unroll 1
+  for (int it = 0; it < 2; ++it) {
+    const int pix0 = blk * PIX + warp * 8 + it * 4;
+    float4 hv[4][NCHUNK];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+      for (int k = 0; k < NCHUNK; ++k)
+        hv[q][k] = (pix0 + q < plane)
+                       ? __ldg(reinterpret_cast<const float4*>(h_img + (size_t)(pix0 + q) * CH + k * 128) + lane)
+                       : make_float4(0.f, 0.f, 0.f, 0.f);
+    float v[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = 0.0f;
+#pragma unroll
+    for (int k = 0; k < NCHUNK; ++k) {
+#pragma unroll
+      for (int tt = 0; tt < TT_MAX_TOOLS; ++tt) {
+        const float4 w = *(reinterpret_cast<const float4*>(s_w + tt * CH + k * 128) + lane);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          float a = v[q * 8 + tt];
+          a = fmaf(hv[q][k].x, w.x, a);
+          a = fmaf(hv[q][k].y, w.y, a);
+          a = fmaf(hv[q][k].z, w.z, a);
+          a = fmaf(hv[q][k].w, w.w, a);
+          v[q * 8 + tt] = a;
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        gap[k * 4 + 0] += hv[q][k].x;
+        gap[k * 4 + 1] += hv[q][k].y;
+        gap[k * 4 + 2] += hv[q][k].z;
+        gap[k * 4 + 3] += hv[q][k].w;
+      }
+    }
+    // transposing butterfly: after the round with offset d a lane keeps the half of its values
+    // selected by its own bit d; five rounds leave value index == lane
+#pragma unroll
+    for (int d = 16, half = 16; d >= 1; d >>= 1, half >>= 1) {
+      const bool upper = (lane & d) != 0;
+#pragma unroll
+      for (int j = 0; j < half; ++j) {
+        const float send = upper ? v[j] : v[j + half];
+        const float keep = upper ? v[j + half] : v[j];
+        v[j] = keep + __shfl_xor_sync(0xffffffffu, send, d);
+      }
+    }
+    const int pix = pix0 + slot;
+    const bool live = (pix < plane) && (t < T);
+    const float z = v[0] + bias;
+    const float pr = sigmoid_acc(z);
+    const bool m = live && (z > p.zthr);
+    if (live) {
+      const size_t o = ((size_t)n * T + t) * plane + pix;
+      p.logits[o] = z;
+      p.probs[o] = pr;
+      p.masks[o] = m ? 1 : 0;
+      sp += pr;
+    }
+    if (m) {
+      cnt += 1;
+      sx += pix % p.Wm;
+      sy += pix / p.Wm;
+    }
+    const uint32_t ballot = __ballot_sync(0xffffffffu, m);
+    if (p.bits && lane < 4 && pix0 + lane < plane) p.bits[(size_t)n * plane + pix0 + lane] = (uint8_t)(ballot >> (8 * lane));
+  }
+
+  // pixel slots -> one value per tool (lanes 0..7), then the 8 warps in order
+#pragma unroll
+  for (int d = 8; d <= 16; d <<= 1) {
+    cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+    sx += __shfl_xor_sync(0xffffffffu, sx, d);
+    sy += __shfl_xor_sync(0xffffffffu, sy, d);
+    sp += __shfl_xor_sync(0xffffffffu, sp, d);
+  }
+  if (lane < TT_MAX_TOOLS) {
+    s_red_i[(warp * TT_MAX_TOOLS + lane) * 3 + 0] = cnt;
+    s_red_i[(warp * TT_MAX_TOOLS + lane) * 3 + 1] = sx;
+    s_red_i[(warp * TT_MAX_TOOLS + lane) * 3 + 2] = sy;
+    s_red_f[warp * TT_MAX_TOOLS + lane] = sp;
+  }
+  if (p.conf_mode == TT_CONF_GAP_LINEAR) {
+#pragma unroll
+    for (int k = 0; k < NCHUNK; ++k)
+      *(reinterpret_cast<float4*>(&s_gapw[warp][k * 128]) + lane) = make_float4(gap[k * 4], gap[k * 4 + 1], gap[k * 4 + 2], gap[k * 4 + 3]);
+  }
+  __syncthreads();
+
+  const ScratchLayout sl = scratch_layout(p.K, plane, CH, T);
+  uint8_t* scr = reinterpret_cast<uint8_t*>(p.scratch);
+  int32_t* part_i = reinterpret_cast<int32_t*>(scr + sl.off_int) + (size_t)blockIdx.x * TT_MAX_TOOLS * 4;
+  float* part_p = reinterpret_cast<float*>(scr + sl.off_p) + (size_t)blockIdx.x * TT_MAX_TOOLS;
+  float* part_h = reinterpret_cast<float*>(scr + sl.off_h) + (size_t)blockIdx.x * CH;
+  if (tid < T) {
+    int c = 0, x = 0, y = 0;
+    float f = 0.0f;
+    for (int w = 0; w < 8; ++w) {
+      c += s_red_i[(w * TT_MAX_TOOLS + tid) * 3 + 0];
+      x += s_red_i[(w * TT_MAX_TOOLS + tid) * 3 + 1];
+      y += s_red_i[(w * TT_MAX_TOOLS + tid) * 3 + 2];
+      f += s_red_f[w * TT_MAX_TOOLS + tid];
+    }
+    part_i[tid * 4 + 0] = c;
+    part_i[tid * 4 + 1] = x;
+    part_i[tid * 4 + 2] = y;
+    part_i[tid * 4 + 3] = 0;
+    part_p[tid] = f;
+  }
+  if (p.conf_mode == TT_CONF_GAP_LINEAR) {
+    for (int c = tid; c < CH; c += POST_THREADS) {
+      float a = 0.0f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) a += s_gapw[w][c];
+      part_h[c] = a;
+    }
+  }
+}
+
 // One block of 1024 threads per stream.  Pooled hidden state: the tile blocks are split into
 // G = 1024 / Ch interleaved groups, thread (g, c) adds channel c over group g's blocks in
 // order, and the G group sums are added in order.  Tool statistics: warp t reduces the partials
@@ -282,7 +436,12 @@ cudaError_t post_prepare() {
 cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s) {
   const int plane = p.Hm * p.Wm;
   const int nb = post_blocks_per_img(plane);
-  post_tile_kernel<<<p.K * nb, POST_THREADS, post_smem_bytes(p.Ch), s>>>(p);
+  const bool direct = p.channels_last && (p.Ch == 128 || p.Ch == 256 || p.Ch == 512) &&
+                      (((uintptr_t)p.h & 15) == 0) && ((p.img_stride & 3) == 0);
+  if (direct && p.Ch == 128) post_direct_kernel<1><<<p.K * nb, POST_THREADS, 0, s>>>(p);
+  else if (direct && p.Ch == 256) post_direct_kernel<2><<<p.K * nb, POST_THREADS, 0, s>>>(p);
+  else if (direct) post_direct_kernel<4><<<p.K * nb, POST_THREADS, 0, s>>>(p);
+  else post_tile_kernel<<<p.K * nb, POST_THREADS, post_smem_bytes(p.Ch), s>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   post_finalize_kernel<<<p.K, FIN_THREADS, 0, s>>>(p);

@@ -109,6 +109,8 @@ struct tt_ctx {
 
   ConvFirstParams first{};      // bf16 path, first encoder layer when its width is supported
   bool use_first = false;
+  ConvFirstTcParams first_tc{}; // ... on the tensor cores when its width allows
+  bool use_first_tc = false;
   SimtLayer simt_enc[TT_MAX_ENC];
   SimtLayer simt_lstm;
   TcLayer tc_enc[TT_MAX_ENC];
@@ -428,7 +430,23 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
       return st;
   } else {
     if (ctx->lay_c[1] % 8) return fail(ctx, TT_ERR_UNSUPPORTED, "bf16 path needs enc_cout[0] in multiples of 8");
-    if (conv_first_supported(ctx->lay_c[1])) {
+    if (conv_first_tc_supported(ctx->lay_c[1])) {
+      const int co = ctx->lay_c[1];
+      std::vector<uint16_t> wb((size_t)co * 27), packed((size_t)co * 32);
+      for (size_t i = 0; i < wb.size(); ++i) wb[i] = f32_to_bf16_rne(w->enc_w[0][i]);
+      conv_first_tc_pack(wb.data(), co, packed.data());
+      std::vector<float> hb(w->enc_b[0], w->enc_b[0] + co);
+      uint16_t* dw = nullptr;
+      float* db = nullptr;
+      if ((st = upload(ctx, &dw, packed)) != TT_OK) return st;
+      if ((st = upload(ctx, &db, hb)) != TT_OK) return st;
+      ConvFirstTcParams& f = ctx->first_tc;
+      f.in = ctx->pre; f.out = reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[0]);
+      f.H = c.net_h; f.W = c.net_w; f.Ho = ctx->lay_h[1]; f.Wo = ctx->lay_w[1]; f.stride = c.enc_stride[0]; f.cout = co;
+      f.tiles_x = (f.Wo + 15) / 16; f.tiles_y = (f.Ho + 7) / 8;
+      f.w_packed = dw; f.bias = db; f.status = ctx->status_dev;
+      ctx->use_first_tc = true;
+    } else if (conv_first_supported(ctx->lay_c[1])) {
       ConvFirstParams& f = ctx->first;
       const int co = ctx->lay_c[1];
       f.in = ctx->pre; f.out = reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[0]);
@@ -545,7 +563,11 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
     TT_CUDA(ctx, launch_conv_simt(q, s));
     if ((ms_ = mark_stage(ctx, TT_STAGE_CONVLSTM, 1)) != TT_OK) return ms_;
   } else {
-    if (ctx->use_first) {
+    if (ctx->use_first_tc) {
+      ctx->first_tc.K = K;
+      TT_CUDA(ctx, launch_conv_first_tc(ctx->first_tc, ctx->sm_count, s));
+      if ((ms_ = mark_stage(ctx, TT_STAGE_ENC0, 1)) != TT_OK) return ms_;
+    } else if (ctx->use_first) {
       ctx->first.K = K;
       TT_CUDA(ctx, launch_conv_first(ctx->first, s));
       if ((ms_ = mark_stage(ctx, TT_STAGE_ENC0, 1)) != TT_OK) return ms_;

@@ -69,6 +69,19 @@ struct ConvFirstParams {
 bool conv_first_supported(int cout);
 cudaError_t launch_conv_first(const ConvFirstParams& p, cudaStream_t s);
 
+// Same layer on the tensor cores (cout 32 or 64): operand tiles are built by gather threads.
+struct ConvFirstTcParams {
+  const float* in;            // [K][3][H][W] fp32
+  __nv_bfloat16* out;         // [K][Ho][Wo][cout] bf16
+  int32_t H, W, Ho, Wo, stride, K, cout, tiles_x, tiles_y;
+  const uint16_t* w_packed;   // device, cout*32 bf16 in the MMA operand layout
+  const float* bias;          // device, [cout]
+  int32_t* status;
+};
+bool conv_first_tc_supported(int cout);
+void conv_first_tc_pack(const uint16_t* w_bf16, int cout, uint16_t* packed);
+cudaError_t launch_conv_first_tc(const ConvFirstTcParams& p, int sm_count, cudaStream_t s);
+
 // ------------------------------------------------- S2/S3 tcgen05 implicit-GEMM conv (bf16)
 // One launch description; tensor maps live in device-visible constant storage owned by the
 // caller (passed by value as __grid_constant__ kernel parameters).
