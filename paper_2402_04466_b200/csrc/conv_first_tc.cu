@@ -3,12 +3,17 @@
 //
 // K = 27 (padded to 32) makes the arithmetic free on tcgen05; the layer is then bound by HBM
 // (read the fp32 input once, write the bf16 output once).  The A operand cannot come from TMA
-// (planar fp32 source, 3 channels), so four producer warps build it: each thread gathers the
-// 27 taps of one output pixel, rounds them to bf16 and writes one 64-byte row of the
+// (planar fp32 source, 3 channels), so four producer warps build it: they first copy the input
+// patch of the tile (all three planes, with halo, zero-filled outside the image) into shared
+// memory with coalesced loads -- the loads of the next tile are already in flight while the
+// current one is being used -- then each thread picks the 27 taps of one output pixel from
+// shared memory, rounds them to bf16 and writes one 64-byte row of the
 // [128 pixels][32] operand tile in the no-swizzle K-major core-matrix layout (8 rows x 16 bytes
 // contiguous; neighbouring core matrices 128 bytes apart along K, 512 bytes apart along M).
 // One warp issues two M128 x COUT x K16 MMAs per tile; four warps run the bias + ReLU epilogue
-// from TMEM.  The operand ring has 4 stages and the accumulator 2 buffers, so gather, MMA and
+// from TMEM, write the bf16 tile into shared memory in the swizzled box layout and hand it to one
+// TMA tile store (full 128-byte lines to L2 instead of 16-byte pieces per thread; the part of a
+// border tile outside the image is clipped by the TMA unit).  The operand ring has 3 stages and the accumulator 2 buffers, so gather, MMA and
 // epilogue of different tiles overlap.  All waits are bounded (see tc_ptx.cuh).
 #include "tt_internal.h"
 #include "tc_ptx.cuh"
@@ -18,15 +23,21 @@ namespace {
 
 using namespace tc;
 
-constexpr int F_STAGES = 4;
+constexpr int F_STAGES = 3;
 constexpr int F_A_BYTES = 128 * 64;                 // 128 rows x 32 bf16
 constexpr int F_THREADS = 288;                      // warps 0-3 gather, 4 MMA, 5-8 epilogue
 constexpr int F_TMEM_COLS = 128;                    // two accumulator buffers of up to 64 columns
 
-template <int COUT>
-__global__ void __launch_bounds__(F_THREADS) conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
-  __shared__ __align__(1024) uint8_t s_a[F_STAGES * F_A_BYTES];
-  __shared__ __align__(1024) uint8_t s_b[COUT * 64];
+template <int COUT, int STRIDE>
+__global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
+  constexpr int PH = 7 * STRIDE + 3, PW = 15 * STRIDE + 3;   // input patch of a 16 x 8 output tile
+  constexpr int PATCH = 3 * PH * PW;
+  constexpr int NPF = (PATCH + 127) / 128;                   // patch elements per producer thread
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* s_out = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);  // one output tile, TMA box layout
+  uint8_t* s_a = s_out + 128 * COUT * 2;                      // operand ring
+  uint8_t* s_b = s_a + F_STAGES * F_A_BYTES;                  // weights in operand layout
+  float (*s_patch)[PATCH] = reinterpret_cast<float (*)[PATCH]>(s_b + COUT * 64);  // [2][PATCH]
   __shared__ __align__(8) uint64_t s_bar[2 * F_STAGES + 4];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
@@ -69,29 +80,54 @@ __global__ void __launch_bounds__(F_THREADS) conv_first_tc_kernel(const __grid_c
   const size_t in_plane = (size_t)p.H * p.W;
 
   if (warp < 4) {
-    // ------------------------------------------------------------------ gather producers
-    const int row = warp * 32 + lane;
+    // ------------------------------------------------------------------ operand producers
+    const int ptid = threadIdx.x;                 // 0..127
+    const int row = ptid;
     const int py = row >> 4, px = row & 15;
     uint8_t* my_row = s_a + (row >> 3) * 512 + (row & 7) * 16;   // + kc * 128 per 16-byte chunk
     uint32_t stage = 0, phase = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    int buf = 0;
+    float pf[NPF];
+
+    // coalesced fetch of one tile's input patch into registers (zero outside the image)
+    auto fetch_patch = [&](int tile) {
       const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, img = tile / tiles_per_img;
-      const int xo = tx * 16 + px, yo = ty * 8 + py;
-      const bool valid = xo < p.Wo && yo < p.Ho;
       const float* src = p.in + (size_t)img * 3 * in_plane;
-      const int x0 = xo * p.stride - 1, y0 = yo * p.stride - 1;
+      const int x_in0 = tx * 16 * STRIDE - 1, y_in0 = ty * 8 * STRIDE - 1;
+#pragma unroll
+      for (int i = 0; i < NPF; ++i) {
+        const int f = ptid + i * 128;
+        const int c = f / (PH * PW), r = (f / PW) % PH, col = f % PW;
+        const int yi = y_in0 + r, xi = x_in0 + col;
+        const bool ok = f < PATCH && yi >= 0 && yi < p.H && xi >= 0 && xi < p.W;
+        pf[i] = ok ? __ldg(src + (size_t)c * in_plane + (size_t)yi * p.W + xi) : 0.0f;
+      }
+    };
+
+    bool fail = false;   // a bounded wait ran out; the four warps learn of it together at the barrier
+    if (blockIdx.x < total_tiles) fetch_patch(blockIdx.x);
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+#pragma unroll
+      for (int i = 0; i < NPF; ++i) {
+        const int f = ptid + i * 128;
+        if (f < PATCH) s_patch[buf][f] = pf[i];
+      }
+      // the four producer warps meet here; with two patch buffers one barrier per tile is enough
+      if (named_barrier_or(1, 128, fail)) break;
+      if (tile + gridDim.x < total_tiles) fetch_patch(tile + gridDim.x);   // next tile's loads fly during the build
       float v[27];
 #pragma unroll
       for (int c = 0; c < 3; ++c)
 #pragma unroll
         for (int ky = 0; ky < 3; ++ky)
 #pragma unroll
-          for (int kx = 0; kx < 3; ++kx) {
-            const int yi = y0 + ky, xi = x0 + kx;
-            const bool ok = valid && yi >= 0 && yi < p.H && xi >= 0 && xi < p.W;
-            v[(c * 3 + ky) * 3 + kx] = ok ? __ldg(src + (size_t)c * in_plane + (size_t)yi * p.W + xi) : 0.0f;
-          }
-      if (!mbar_wait(smem_u32(a_empty + stage), phase ^ 1u, abort_flag, p.status, 0x500 + (int)stage)) break;
+          for (int kx = 0; kx < 3; ++kx)
+            v[(c * 3 + ky) * 3 + kx] = s_patch[buf][(c * PH + py * STRIDE + ky) * PW + px * STRIDE + kx];
+      buf ^= 1;
+      if (!mbar_wait(smem_u32(a_empty + stage), phase ^ 1u, abort_flag, p.status, 0x500 + (int)stage)) {
+        fail = true;
+        continue;
+      }
       uint8_t* dst = my_row + stage * F_A_BYTES;
       uint4 u;
       u.x = pack_bf16(v[0], v[1]);   u.y = pack_bf16(v[2], v[3]);   u.z = pack_bf16(v[4], v[5]);   u.w = pack_bf16(v[6], v[7]);
@@ -134,41 +170,52 @@ __global__ void __launch_bounds__(F_THREADS) conv_first_tc_kernel(const __grid_c
   } else {
     // --------------------------------------------------------------------------- epilogue
     const int quarter = warp & 3;
-    const int row = quarter * 32 + lane;
-    const int py = row >> 4, px = row & 15;
+    const int row = quarter * 32 + lane;            // tile row = pixel (row / 16, row % 16) of the patch
+    const bool leader = (warp == 5 && lane == 0);   // issues and tracks the TMA stores
+    constexpr int ROW_BYTES = COUT * 2;             // 128 (128-byte swizzle) or 64 (64-byte swizzle)
+    const uint32_t sw = ROW_BYTES == 128 ? (uint32_t)(row & 7) : (uint32_t)((row >> 1) & 3);
+    uint8_t* my_out = s_out + row * ROW_BYTES;
     uint32_t acc_phase = 0;
     int acc = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
       const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, img = tile / tiles_per_img;
-      const int xo = tx * 16 + px, yo = ty * 8 + py;
-      const bool valid = xo < p.Wo && yo < p.Ho;
-      if (!mbar_wait(smem_u32(t_full + acc), acc_phase, abort_flag, p.status, 0x800 + acc)) break;
+      const bool fail = !mbar_wait(smem_u32(t_full + acc), acc_phase, abort_flag, p.status, 0x800 + acc);
+      // the previous tile's store must have finished reading s_out before it is overwritten
+      if (leader) bulk_wait_group_read0();
+      if (named_barrier_or(2, 128, fail)) break;   // all four warps stop together if any wait ran out
       tc_fence_after();
       const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 64);
-      __nv_bfloat16* dst = p.out + (((size_t)img * p.Ho + yo) * p.Wo + xo) * COUT;
 #pragma unroll
       for (int ck = 0; ck < COUT / 32; ++ck) {
         uint32_t v[32];
         tmem_ld32(t_addr + (uint32_t)(ck * 32), v);
-        if (valid) {
-          const float4* b4 = reinterpret_cast<const float4*>(p.bias + ck * 32);
 #pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            const float4 ba = __ldg(b4 + i / 4), bb = __ldg(b4 + i / 4 + 1);
-            uint4 u;
-            u.x = pack_bf16(fmaxf(__uint_as_float(v[i + 0]) + ba.x, 0.f), fmaxf(__uint_as_float(v[i + 1]) + ba.y, 0.f));
-            u.y = pack_bf16(fmaxf(__uint_as_float(v[i + 2]) + ba.z, 0.f), fmaxf(__uint_as_float(v[i + 3]) + ba.w, 0.f));
-            u.z = pack_bf16(fmaxf(__uint_as_float(v[i + 4]) + bb.x, 0.f), fmaxf(__uint_as_float(v[i + 5]) + bb.y, 0.f));
-            u.w = pack_bf16(fmaxf(__uint_as_float(v[i + 6]) + bb.z, 0.f), fmaxf(__uint_as_float(v[i + 7]) + bb.w, 0.f));
-            *reinterpret_cast<uint4*>(dst + ck * 32 + i) = u;
-          }
+        for (int i = 0; i < 32; i += 8) {
+          const float4 ba = __ldg(reinterpret_cast<const float4*>(p.bias + ck * 32 + i));
+          const float4 bb = __ldg(reinterpret_cast<const float4*>(p.bias + ck * 32 + i + 4));
+          uint4 u;
+          u.x = pack_bf16(fmaxf(__uint_as_float(v[i + 0]) + ba.x, 0.f), fmaxf(__uint_as_float(v[i + 1]) + ba.y, 0.f));
+          u.y = pack_bf16(fmaxf(__uint_as_float(v[i + 2]) + ba.z, 0.f), fmaxf(__uint_as_float(v[i + 3]) + ba.w, 0.f));
+          u.z = pack_bf16(fmaxf(__uint_as_float(v[i + 4]) + bb.x, 0.f), fmaxf(__uint_as_float(v[i + 5]) + bb.y, 0.f));
+          u.w = pack_bf16(fmaxf(__uint_as_float(v[i + 6]) + bb.z, 0.f), fmaxf(__uint_as_float(v[i + 7]) + bb.w, 0.f));
+          // 16-byte chunk c of this row sits at chunk position c ^ sw of the swizzled box
+          const uint32_t c = (uint32_t)(ck * 4 + (i >> 3));
+          *reinterpret_cast<uint4*>(my_out + ((c ^ sw) << 4)) = u;
         }
       }
+      // the accumulator has been read: hand the TMEM buffer back to the MMA warp
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(t_empty + acc));
+      fence_proxy_async_smem();
+      asm volatile("bar.sync 3, 128;" ::: "memory");
+      if (leader) {
+        tma_store_4d(&p.map_out, smem_u32(s_out), 0, tx * 16, ty * 8, img);
+        bulk_commit_group();
+      }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
+    if (leader) bulk_wait_group0();
   }
 
   __syncwarp();
@@ -182,6 +229,17 @@ __global__ void __launch_bounds__(F_THREADS) conv_first_tc_kernel(const __grid_c
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)F_TMEM_COLS)
                  : "memory");
   }
+}
+
+template <int COUT, int STRIDE>
+cudaError_t launch_t(const ConvFirstTcParams& p, int grid, cudaStream_t s) {
+  constexpr int PH = 7 * STRIDE + 3, PW = 15 * STRIDE + 3;
+  constexpr int SMEM = 1024 + 128 * COUT * 2 + F_STAGES * F_A_BYTES + COUT * 64 + 2 * 3 * PH * PW * 4;
+  auto kern = conv_first_tc_kernel<COUT, STRIDE>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  if (e != cudaSuccess) return e;
+  kern<<<grid, F_THREADS, SMEM, s>>>(p);
+  return cudaGetLastError();
 }
 
 }  // namespace
@@ -198,10 +256,11 @@ void conv_first_tc_pack(const uint16_t* w_bf16, int cout, uint16_t* packed) {
 cudaError_t launch_conv_first_tc(const ConvFirstTcParams& p, int sm_count, cudaStream_t s) {
   const int total = p.K * p.tiles_x * p.tiles_y;
   const int grid = total < 3 * sm_count ? total : 3 * sm_count;
-  if (p.cout == 32) conv_first_tc_kernel<32><<<grid, F_THREADS, 0, s>>>(p);
-  else if (p.cout == 64) conv_first_tc_kernel<64><<<grid, F_THREADS, 0, s>>>(p);
-  else return cudaErrorInvalidValue;
-  return cudaGetLastError();
+  if (p.cout == 32 && p.stride == 1) return launch_t<32, 1>(p, grid, s);
+  if (p.cout == 32 && p.stride == 2) return launch_t<32, 2>(p, grid, s);
+  if (p.cout == 64 && p.stride == 1) return launch_t<64, 1>(p, grid, s);
+  if (p.cout == 64 && p.stride == 2) return launch_t<64, 2>(p, grid, s);
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace tt

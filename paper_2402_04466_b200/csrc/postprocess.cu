@@ -183,8 +183,10 @@ __global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const __grid_co
 template <int NCHUNK>
 __global__ void __launch_bounds__(POST_THREADS) post_direct_kernel(const __grid_constant__ PostParams p) {
   constexpr int CH = NCHUNK * 128;
-  __shared__ __align__(16) float s_w[TT_MAX_TOOLS * CH];
-  __shared__ __align__(16) float s_gapw[8][CH];
+  extern __shared__ __align__(16) float s_dyn[];
+  float* s_h = s_dyn;                         // [8 warps][8 pixels][CH]: each warp's pixels, filled by cp.async
+  float* s_w = s_h + PIX * CH;                // [TT_MAX_TOOLS][CH]
+  float (*s_gapw)[CH] = reinterpret_cast<float (*)[CH]>(s_w + TT_MAX_TOOLS * CH);  // [8][CH]
   __shared__ float s_red_f[8 * TT_MAX_TOOLS];
   __shared__ int s_red_i[8 * TT_MAX_TOOLS * 3];
 
@@ -195,8 +197,29 @@ __global__ void __launch_bounds__(POST_THREADS) post_direct_kernel(const __grid_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const float* h_img = p.h + (size_t)p.idx.v[n] * p.img_stride;
 
+  // Every lane copies, for each of its warp's 8 pixels, the 16 bytes per 128-channel chunk that it
+  // will consume itself: the copies need no registers, are all in flight at once, and a lane only
+  // ever reads back what it copied, so waiting for its own copies is the only synchronisation.
+  float* my_h = s_h + (size_t)warp * 8 * CH;
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const int pix = blk * PIX + warp * 8 + q;
+#pragma unroll
+    for (int k = 0; k < NCHUNK; ++k) {
+      float* dst = my_h + q * CH + k * 128 + lane * 4;
+      if (pix < plane) {
+        const float* src = h_img + (size_t)pix * CH + k * 128 + lane * 4;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+      } else {
+        *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+
   for (int i = tid; i < TT_MAX_TOOLS * CH; i += POST_THREADS) s_w[i] = i < T * CH ? __ldg(p.head_w + i) : 0.0f;
   __syncthreads();
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
 
   const int slot = lane >> 3, t = lane & 7;       // after the butterfly this lane owns (pixel slot, tool)
   const float bias = t < T ? __ldg(p.head_b + t) : 0.0f;
@@ -214,9 +237,7 @@ __global__ void __launch_bounds__(POST_THREADS) post_direct_kernel(const __grid_
     for (int q = 0; q < 4; ++q)
 #pragma unroll
       for (int k = 0; k < NCHUNK; ++k)
-        hv[q][k] = (pix0 + q < plane)
-                       ? __ldg(reinterpret_cast<const float4*>(h_img + (size_t)(pix0 + q) * CH + k * 128) + lane)
-                       : make_float4(0.f, 0.f, 0.f, 0.f);
+        hv[q][k] = *reinterpret_cast<const float4*>(my_h + (it * 4 + q) * CH + k * 128 + lane * 4);
     float v[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = 0.0f;
@@ -352,7 +373,7 @@ __global__ void __launch_bounds__(FIN_THREADS) post_finalize_kernel(const __grid
     const int g = tid / Ch, c = tid - g * Ch;
     float s = 0.0f;
     if (g < G) {
-#pragma unroll 8
+#pragma unroll 32
       for (int b = g; b < nb; b += G) s += part_h[(size_t)b * Ch + c];
     }
     s_part[tid] = s;
@@ -368,6 +389,7 @@ __global__ void __launch_bounds__(FIN_THREADS) post_finalize_kernel(const __grid
     const int t = warp;
     long long cnt = 0, sx = 0, sy = 0;
     float sp = 0.0f;
+#pragma unroll 8
     for (int b = lane; b < nb; b += 32) {
       const int4 v = part_i[(size_t)b * TT_MAX_TOOLS + t];
       cnt += v.x; sx += v.y; sy += v.z;
@@ -430,7 +452,14 @@ cudaError_t post_static_scratch(void** ptr) {
 }
 
 cudaError_t post_prepare() {
-  return cudaFuncSetAttribute(post_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)post_smem_bytes(512));
+  cudaError_t e = cudaFuncSetAttribute(post_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)post_smem_bytes(512));
+  if (e != cudaSuccess) return e;
+  const int per_ch = (PIX + TT_MAX_TOOLS + 8) * (int)sizeof(float);
+  e = cudaFuncSetAttribute(post_direct_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, per_ch * 128);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(post_direct_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, per_ch * 256);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(post_direct_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, per_ch * 512);
 }
 
 cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s) {
@@ -438,9 +467,10 @@ cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s) {
   const int nb = post_blocks_per_img(plane);
   const bool direct = p.channels_last && (p.Ch == 128 || p.Ch == 256 || p.Ch == 512) &&
                       (((uintptr_t)p.h & 15) == 0) && ((p.img_stride & 3) == 0);
-  if (direct && p.Ch == 128) post_direct_kernel<1><<<p.K * nb, POST_THREADS, 0, s>>>(p);
-  else if (direct && p.Ch == 256) post_direct_kernel<2><<<p.K * nb, POST_THREADS, 0, s>>>(p);
-  else if (direct) post_direct_kernel<4><<<p.K * nb, POST_THREADS, 0, s>>>(p);
+  const size_t dsm = (size_t)(PIX + TT_MAX_TOOLS + 8) * p.Ch * sizeof(float);
+  if (direct && p.Ch == 128) post_direct_kernel<1><<<p.K * nb, POST_THREADS, dsm, s>>>(p);
+  else if (direct && p.Ch == 256) post_direct_kernel<2><<<p.K * nb, POST_THREADS, dsm, s>>>(p);
+  else if (direct) post_direct_kernel<4><<<p.K * nb, POST_THREADS, dsm, s>>>(p);
   else post_tile_kernel<<<p.K * nb, POST_THREADS, post_smem_bytes(p.Ch), s>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;

@@ -445,6 +445,12 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
       f.H = c.net_h; f.W = c.net_w; f.Ho = ctx->lay_h[1]; f.Wo = ctx->lay_w[1]; f.stride = c.enc_stride[0]; f.cout = co;
       f.tiles_x = (f.Wo + 15) / 16; f.tiles_y = (f.Ho + 7) / 8;
       f.w_packed = dw; f.bias = db; f.status = ctx->status_dev;
+      {
+        const cuuint64_t dims[4] = {(cuuint64_t)co, (cuuint64_t)f.Wo, (cuuint64_t)f.Ho, (cuuint64_t)S};
+        const cuuint64_t str[3] = {(cuuint64_t)co * 2, (cuuint64_t)f.Wo * co * 2, (cuuint64_t)f.Ho * f.Wo * co * 2};
+        const cuuint32_t box[4] = {(cuuint32_t)co, 16, 8, 1};
+        if ((st = encode_map(ctx, &f.map_out, ctx->enc_out[0], 4, dims, str, box, co * 2)) != TT_OK) return st;
+      }
       ctx->use_first_tc = true;
     } else if (conv_first_supported(ctx->lay_c[1])) {
       ConvFirstParams& f = ctx->first;

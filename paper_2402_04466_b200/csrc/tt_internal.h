@@ -56,6 +56,11 @@ struct ConvSimtParams {
 };
 cudaError_t launch_conv_simt(const ConvSimtParams& p, cudaStream_t s);
 
+// Opaque 128-byte TMA tensor map, passed inside __grid_constant__ kernel parameters.
+struct alignas(64) TensorMap128 {
+  uint8_t bytes[128];
+};
+
 // --------------------------------------- S2 first encoder layer of the bf16 path (Cin = 3)
 // Passed by value: the weights sit in the kernel parameter block (constant bank).
 constexpr int CONV_FIRST_MAX_COUT = 64;
@@ -71,6 +76,7 @@ cudaError_t launch_conv_first(const ConvFirstParams& p, cudaStream_t s);
 
 // Same layer on the tensor cores (cout 32 or 64): operand tiles are built by gather threads.
 struct ConvFirstTcParams {
+  TensorMap128 map_out;       // output [K][Ho][Wo][cout] bf16, box [cout][16][8][1], 128B / 64B swizzle
   const float* in;            // [K][3][H][W] fp32
   __nv_bfloat16* out;         // [K][Ho][Wo][cout] bf16
   int32_t H, W, Ho, Wo, stride, K, cout, tiles_x, tiles_y;
@@ -85,10 +91,6 @@ cudaError_t launch_conv_first_tc(const ConvFirstTcParams& p, int sm_count, cudaS
 // ------------------------------------------------- S2/S3 tcgen05 implicit-GEMM conv (bf16)
 // One launch description; tensor maps live in device-visible constant storage owned by the
 // caller (passed by value as __grid_constant__ kernel parameters).
-struct alignas(64) TensorMap128 {
-  uint8_t bytes[128];
-};
-
 enum TcEpilogue : int32_t { TC_EPI_RELU_BF16 = 0, TC_EPI_LSTM = 1 };
 
 struct ConvTcParams {
