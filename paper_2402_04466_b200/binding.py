@@ -195,7 +195,8 @@ class Context:
         _check(self.lib, self.lib.tt_map_size(self.handle, C.byref(hm), C.byref(wm)), self.handle)
         self.hm, self.wm = hm.value, wm.value
         self.n_tools, self.hidden = cfg.n_tools, cfg.hidden
-        self._last_k = 0
+        self._ks = []                # stream counts of the submits in flight, oldest first
+        self._inflight_keep = []     # keeps the frame tensors of in-flight submits alive
 
     # -- lifetime
     def destroy(self):
@@ -244,25 +245,31 @@ class Context:
         sts = (C.c_void_p * max(K, 1))(*[s.value if isinstance(s, C.c_void_p) else s for s in states])
         st = self.lib.tt_submit_frames(self.handle, K, fr, sts)
         _check(self.lib, st, self.handle)
-        self._last_k = K
-        self._inflight_keep = list(frames)
+        self._ks.append(K)
+        self._inflight_keep.append(list(frames))
 
     def submit_raw(self, K: int, frame_array, state_array) -> int:
         """Pre-marshalled arrays (tt_frame[K], void*[K]); returns the status without raising."""
         st = self.lib.tt_submit_frames(self.handle, K, frame_array, state_array)
         if st == TT_OK:
-            self._last_k = K
+            self._ks.append(K)
+            self._inflight_keep.append(None)
         return st
 
     def sync(self) -> List[Dict]:
         res = (tt_result * TT_MAX_STREAMS)()
         st = self.lib.tt_sync(self.handle, res)
         _check(self.lib, st, self.handle)
-        self._inflight_keep = None
-        return [_result_to_dict(res[k], self.n_tools) for k in range(self._last_k)]
+        k_done = self._ks.pop(0)                 # submits complete oldest first
+        self._inflight_keep.pop(0)
+        return [_result_to_dict(res[k], self.n_tools) for k in range(k_done)]
 
     def sync_raw(self, result_array) -> int:
-        return self.lib.tt_sync(self.handle, result_array)
+        st = self.lib.tt_sync(self.handle, result_array)
+        if st == TT_OK and self._ks:
+            self._ks.pop(0)
+            self._inflight_keep.pop(0)
+        return st
 
     def set_profiling(self, on: bool):
         _check(self.lib, self.lib.tt_set_profiling(self.handle, int(on)), self.handle)

@@ -117,7 +117,29 @@ struct tt_ctx {
   TcLayer tc_lstm;
 
   tt_state states[TT_MAX_STREAMS];
-  bool in_flight = false;
+  // Up to two submits may be in flight.  Everything a tick owns (frame staging, outputs, result
+  // blocks, events) exists twice; the members above/below named like the slot's are the slot that
+  // is currently bound (bind_slot / save_slot).
+  struct Slot {
+    uint8_t* frames_stage = nullptr;
+    float *logits = nullptr, *probs = nullptr;
+    uint8_t *masks = nullptr, *bits = nullptr, *overlay = nullptr;
+    tt_result *results_dev = nullptr, *results_host = nullptr;
+    int32_t* status_host = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_stop = nullptr, ev_copy = nullptr;
+    cudaEvent_t stage_ev[TT_STAGE_COUNT + 1] = {};
+    bool stage_ran[TT_STAGE_COUNT] = {};
+    bool profiled = false;
+    int K = 0;
+    tt_frame frames[TT_MAX_STREAMS];
+    tt_state* states[TT_MAX_STREAMS];
+  } slots[2];
+  int q_head = 0, q_count = 0;      // oldest in-flight slot, number in flight
+  int bound = 0;                    // slot whose resources the view members hold
+  int last_done = -1;               // slot of the last completed submit (debug taps)
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_copy = nullptr;
+  bool tick_profiled = false;
   int K_inflight = 0;
   tt_frame frames_inflight[TT_MAX_STREAMS];
   tt_state* states_inflight[TT_MAX_STREAMS];
@@ -147,6 +169,31 @@ tt_status fail(tt_ctx* ctx, tt_status st, const char* fmt, ...) {
     g_create_err = buf;
   }
   return st;
+}
+
+void bind_slot(tt_ctx* ctx, int i) {
+  const tt_ctx::Slot& sl = ctx->slots[i];
+  ctx->frames_stage = sl.frames_stage; ctx->logits = sl.logits; ctx->probs = sl.probs; ctx->masks = sl.masks;
+  ctx->bits = sl.bits; ctx->overlay = sl.overlay; ctx->results_dev = sl.results_dev; ctx->results_host = sl.results_host;
+  ctx->status_host = sl.status_host; ctx->ev_start = sl.ev_start; ctx->ev_stop = sl.ev_stop; ctx->ev_copy = sl.ev_copy;
+  for (int k = 0; k <= TT_STAGE_COUNT; ++k) ctx->stage_ev[k] = sl.stage_ev[k];
+  for (int k = 0; k < TT_STAGE_COUNT; ++k) ctx->stage_ran[k] = sl.stage_ran[k];
+  ctx->tick_profiled = sl.profiled;
+  ctx->K_inflight = sl.K;
+  for (int k = 0; k < TT_MAX_STREAMS; ++k) { ctx->frames_inflight[k] = sl.frames[k]; ctx->states_inflight[k] = sl.states[k]; }
+  ctx->bound = i;
+}
+
+void save_slot(tt_ctx* ctx, int i) {
+  tt_ctx::Slot& sl = ctx->slots[i];
+  sl.frames_stage = ctx->frames_stage; sl.logits = ctx->logits; sl.probs = ctx->probs; sl.masks = ctx->masks;
+  sl.bits = ctx->bits; sl.overlay = ctx->overlay; sl.results_dev = ctx->results_dev; sl.results_host = ctx->results_host;
+  sl.status_host = ctx->status_host; sl.ev_start = ctx->ev_start; sl.ev_stop = ctx->ev_stop; sl.ev_copy = ctx->ev_copy;
+  for (int k = 0; k <= TT_STAGE_COUNT; ++k) sl.stage_ev[k] = ctx->stage_ev[k];
+  for (int k = 0; k < TT_STAGE_COUNT; ++k) sl.stage_ran[k] = ctx->stage_ran[k];
+  sl.profiled = ctx->tick_profiled;
+  sl.K = ctx->K_inflight;
+  for (int k = 0; k < TT_MAX_STREAMS; ++k) { sl.frames[k] = ctx->frames_inflight[k]; sl.states[k] = ctx->states_inflight[k]; }
 }
 
 #define TT_CUDA(ctx, expr)                                                                         \
@@ -340,9 +387,7 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
     TT_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->stream, cudaStreamNonBlocking));
     ctx->own_stream = true;
   }
-  TT_CUDA(ctx, cudaEventCreate(&ctx->ev_start));
-  TT_CUDA(ctx, cudaEventCreate(&ctx->ev_stop));
-  for (int i = 0; i <= TT_STAGE_COUNT; ++i) TT_CUDA(ctx, cudaEventCreate(&ctx->stage_ev[i]));
+  TT_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
   for (int i = 0; i < TT_STAGE_COUNT; ++i) ctx->stage_ms[i] = -1.f;
   TT_CUDA(ctx, post_prepare());
 
@@ -363,7 +408,6 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
   ctx->zthr = (float)std::log((double)c.threshold / (1.0 - (double)c.threshold));
 
   tt_status st;
-  if ((st = dev_alloc(ctx, &ctx->frames_stage, (size_t)S * ctx->frame_bytes + 16)) != TT_OK) return st;
   if ((st = dev_alloc(ctx, &ctx->pre, (size_t)S * 3 * c.net_h * c.net_w)) != TT_OK) return st;
   size_t max_floats = (size_t)3 * c.net_h * c.net_w;
   for (int l = 0; l < c.n_enc; ++l) {
@@ -390,21 +434,31 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
   } else {
     if ((st = dev_alloc(ctx, &ctx->h_f32, (size_t)S * 2 * ctx->Ch * plane)) != TT_OK) return st;
   }
-  if ((st = dev_alloc(ctx, &ctx->logits, (size_t)S * ctx->T * plane)) != TT_OK) return st;
-  if ((st = dev_alloc(ctx, &ctx->probs, (size_t)S * ctx->T * plane)) != TT_OK) return st;
-  if ((st = dev_alloc(ctx, &ctx->masks, (size_t)S * ctx->T * plane)) != TT_OK) return st;
-  if ((st = dev_alloc(ctx, &ctx->bits, (size_t)S * plane)) != TT_OK) return st;
-  if (c.overlay && (st = dev_alloc(ctx, &ctx->overlay, (size_t)S * c.src_w * c.src_h * 4)) != TT_OK) return st;
-  if ((st = dev_alloc(ctx, &ctx->results_dev, (size_t)S)) != TT_OK) return st;
   if ((st = dev_alloc(ctx, &ctx->status_dev, 1)) != TT_OK) return st;
   {
     uint8_t* scr = nullptr;
     if ((st = dev_alloc(ctx, &scr, post_scratch_bytes(S, ctx->Hm, ctx->Wm, ctx->Ch, ctx->T))) != TT_OK) return st;
     ctx->post_scratch = scr;
   }
-  TT_CUDA(ctx, cudaHostAlloc(reinterpret_cast<void**>(&ctx->results_host), sizeof(tt_result) * S, cudaHostAllocDefault));
-  TT_CUDA(ctx, cudaHostAlloc(reinterpret_cast<void**>(&ctx->status_host), sizeof(int32_t), cudaHostAllocDefault));
-  *ctx->status_host = 0;
+  // per-slot resources: two submits may be in flight
+  for (int i = 0; i < 2; ++i) {
+    tt_ctx::Slot& sl = ctx->slots[i];
+    if ((st = dev_alloc(ctx, &sl.frames_stage, (size_t)S * ctx->frame_bytes + 16)) != TT_OK) return st;
+    if ((st = dev_alloc(ctx, &sl.logits, (size_t)S * ctx->T * plane)) != TT_OK) return st;
+    if ((st = dev_alloc(ctx, &sl.probs, (size_t)S * ctx->T * plane)) != TT_OK) return st;
+    if ((st = dev_alloc(ctx, &sl.masks, (size_t)S * ctx->T * plane)) != TT_OK) return st;
+    if ((st = dev_alloc(ctx, &sl.bits, (size_t)S * plane)) != TT_OK) return st;
+    if (c.overlay && (st = dev_alloc(ctx, &sl.overlay, (size_t)S * c.src_w * c.src_h * 4)) != TT_OK) return st;
+    if ((st = dev_alloc(ctx, &sl.results_dev, (size_t)S)) != TT_OK) return st;
+    TT_CUDA(ctx, cudaHostAlloc(reinterpret_cast<void**>(&sl.results_host), sizeof(tt_result) * S, cudaHostAllocDefault));
+    TT_CUDA(ctx, cudaHostAlloc(reinterpret_cast<void**>(&sl.status_host), sizeof(int32_t), cudaHostAllocDefault));
+    *sl.status_host = 0;
+    TT_CUDA(ctx, cudaEventCreate(&sl.ev_start));
+    TT_CUDA(ctx, cudaEventCreate(&sl.ev_stop));
+    TT_CUDA(ctx, cudaEventCreateWithFlags(&sl.ev_copy, cudaEventDisableTiming));
+    for (int k = 0; k <= TT_STAGE_COUNT; ++k) TT_CUDA(ctx, cudaEventCreate(&sl.stage_ev[k]));
+  }
+  bind_slot(ctx, 0);
 
   // ---- weights
   const bool r = ctx->bf16;  // round weights to bf16 on the bf16 path
@@ -496,12 +550,18 @@ void release(tt_ctx* ctx) {
   cudaSetDevice(ctx->dev);
   if (ctx->stream) cudaStreamSynchronize(ctx->stream);
   for (void* p : ctx->allocs) cudaFree(p);
-  if (ctx->results_host) cudaFreeHost(ctx->results_host);
-  if (ctx->status_host) cudaFreeHost(ctx->status_host);
-  if (ctx->ev_start) cudaEventDestroy(ctx->ev_start);
-  if (ctx->ev_stop) cudaEventDestroy(ctx->ev_stop);
-  for (int i = 0; i <= TT_STAGE_COUNT; ++i)
-    if (ctx->stage_ev[i]) cudaEventDestroy(ctx->stage_ev[i]);
+  if (ctx->copy_stream) cudaStreamSynchronize(ctx->copy_stream);
+  for (int i = 0; i < 2; ++i) {
+    tt_ctx::Slot& sl = ctx->slots[i];
+    if (sl.results_host) cudaFreeHost(sl.results_host);
+    if (sl.status_host) cudaFreeHost(sl.status_host);
+    if (sl.ev_start) cudaEventDestroy(sl.ev_start);
+    if (sl.ev_stop) cudaEventDestroy(sl.ev_stop);
+    if (sl.ev_copy) cudaEventDestroy(sl.ev_copy);
+    for (int k = 0; k <= TT_STAGE_COUNT; ++k)
+      if (sl.stage_ev[k]) cudaEventDestroy(sl.stage_ev[k]);
+  }
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   if (ctx->own_stream && ctx->stream) cudaStreamDestroy(ctx->stream);
   delete ctx;
 }
@@ -713,7 +773,7 @@ static tt_status zero_state(tt_ctx* ctx, tt_state* st) {
 tt_status tt_state_create(tt_ctx* ctx, tt_state** out) {
   if (!ctx || !out) return TT_ERR_INVALID_ARG;
   *out = nullptr;
-  if (ctx->in_flight) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
+  if (ctx->q_count) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
   for (int i = 0; i < ctx->cfg.max_streams; ++i)
     if (!ctx->states[i].in_use) {
       ctx->states[i].in_use = true;
@@ -727,13 +787,13 @@ tt_status tt_state_create(tt_ctx* ctx, tt_state** out) {
 
 tt_status tt_state_reset(tt_ctx* ctx, tt_state* st) {
   if (!ctx || !owns_state(ctx, st)) return ctx ? fail(ctx, TT_ERR_INVALID_ARG, "state does not belong to this context") : TT_ERR_INVALID_ARG;
-  if (ctx->in_flight) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
+  if (ctx->q_count) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
   return zero_state(ctx, st);
 }
 
 tt_status tt_state_export(tt_ctx* ctx, tt_state* st, float* h_host, float* c_host) {
   if (!ctx || !owns_state(ctx, st) || !h_host || !c_host) return ctx ? fail(ctx, TT_ERR_INVALID_ARG, "bad state or null buffer") : TT_ERR_INVALID_ARG;
-  if (ctx->in_flight) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
+  if (ctx->q_count) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
   TT_CUDA(ctx, cudaSetDevice(ctx->dev));
   const int plane = ctx->Hm * ctx->Wm;
   const size_t n = (size_t)ctx->Ch * plane;
@@ -753,7 +813,7 @@ tt_status tt_state_export(tt_ctx* ctx, tt_state* st, float* h_host, float* c_hos
 
 tt_status tt_state_import(tt_ctx* ctx, tt_state* st, const float* h_host, const float* c_host) {
   if (!ctx || !owns_state(ctx, st) || !h_host || !c_host) return ctx ? fail(ctx, TT_ERR_INVALID_ARG, "bad state or null buffer") : TT_ERR_INVALID_ARG;
-  if (ctx->in_flight) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
+  if (ctx->q_count) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
   TT_CUDA(ctx, cudaSetDevice(ctx->dev));
   const int plane = ctx->Hm * ctx->Wm;
   const size_t n = (size_t)ctx->Ch * plane;
@@ -777,7 +837,7 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
   if (!frames || !states || K < 1) return fail(ctx, TT_ERR_INVALID_ARG, "null frames/states or K < 1");
   if (K > ctx->cfg.max_streams)
     return fail(ctx, TT_ERR_ADMISSION, "K = %d streams exceed the %d this context was sized for", K, ctx->cfg.max_streams);
-  if (ctx->in_flight) return fail(ctx, TT_ERR_NOT_READY, "a submit is already in flight; call tt_sync first");
+  if (ctx->q_count >= 2) return fail(ctx, TT_ERR_NOT_READY, "two submits are already in flight; call tt_sync first");
   for (int n = 0; n < K; ++n) {
     if (!owns_state(ctx, states[n])) return fail(ctx, TT_ERR_INVALID_ARG, "states[%d] is null or belongs to another context", n);
     if (!frames[n].data) return fail(ctx, TT_ERR_INVALID_ARG, "frames[%d].data is null", n);
@@ -785,10 +845,13 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
       if (states[m] == states[n]) return fail(ctx, TT_ERR_INVALID_ARG, "states[%d] and states[%d] are the same state", m, n);
   }
   TT_CUDA(ctx, cudaSetDevice(ctx->dev));
+  const int slot = (ctx->q_head + ctx->q_count) & 1;   // the slot that is not in flight (or the only free one)
+  bind_slot(ctx, slot);
   cudaStream_t s = ctx->stream;
   TT_CUDA(ctx, cudaEventRecord(ctx->ev_start, s));
   for (int i = 0; i < TT_STAGE_COUNT; ++i) ctx->stage_ran[i] = false;
   ctx->stage_valid = false;
+  ctx->tick_profiled = ctx->profiling;
   if (ctx->profiling) TT_CUDA(ctx, cudaEventRecord(ctx->stage_ev[0], s));
   FramePtrs fp{};
   bool any_h2d = false;
@@ -796,14 +859,21 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
     if (frames[n].on_device) {
       fp.p[n] = frames[n].data;
     } else {
+      // host frames go over a copy stream of their own, so the copy of this tick can run while the
+      // previous tick still computes; the compute stream waits for the copy below
       uint8_t* dst = ctx->frames_stage + (size_t)n * ctx->frame_bytes;
-      TT_CUDA(ctx, cudaMemcpyAsync(dst, frames[n].data, ctx->frame_bytes, cudaMemcpyHostToDevice, s));
+      TT_CUDA(ctx, cudaMemcpyAsync(dst, frames[n].data, ctx->frame_bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
       fp.p[n] = dst;
       any_h2d = true;
     }
   }
-  tt_status st = any_h2d ? mark_stage(ctx, TT_STAGE_H2D, 0) : TT_OK;
-  if (st != TT_OK) return st;
+  tt_status st = TT_OK;
+  if (any_h2d) {
+    TT_CUDA(ctx, cudaEventRecord(ctx->ev_copy, ctx->copy_stream));
+    TT_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_copy, 0));
+    st = mark_stage(ctx, TT_STAGE_H2D, 0);
+    if (st != TT_OK) return st;
+  }
   st = enqueue_tick(ctx, K, fp, states);
   if (st != TT_OK) return st;
   TT_CUDA(ctx, cudaMemcpyAsync(ctx->results_host, ctx->results_dev, sizeof(tt_result) * K, cudaMemcpyDeviceToHost, s));
@@ -817,15 +887,18 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
     states[n]->last_pos = n;
   }
   ctx->K_inflight = K;
-  ctx->in_flight = true;
+  save_slot(ctx, slot);
+  ctx->q_count += 1;
   return TT_OK;
 }
 
 tt_status tt_sync(tt_ctx* ctx, tt_result* results) {
   if (!ctx) return TT_ERR_INVALID_ARG;
-  if (!ctx->in_flight) return fail(ctx, TT_ERR_NOT_READY, "nothing has been submitted");
+  if (ctx->q_count == 0) return fail(ctx, TT_ERR_NOT_READY, "nothing has been submitted");
   if (!results) return fail(ctx, TT_ERR_INVALID_ARG, "null results");
   TT_CUDA(ctx, cudaSetDevice(ctx->dev));
+  const int slot = ctx->q_head;
+  bind_slot(ctx, slot);
   if (ctx->cfg.sync_timeout_ns == 0) {
     TT_CUDA(ctx, cudaEventSynchronize(ctx->ev_stop));
   } else {
@@ -839,10 +912,12 @@ tt_status tt_sync(tt_ctx* ctx, tt_result* results) {
       std::this_thread::yield();
     }
   }
-  ctx->in_flight = false;
+  ctx->q_head ^= 1;
+  ctx->q_count -= 1;
+  ctx->last_done = slot;
   float ms = 0.f;
   TT_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->ev_start, ctx->ev_stop));
-  if (ctx->profiling) {
+  if (ctx->tick_profiled) {
     int prev = 0;  // index into stage_ev of the last recorded event
     for (int i = 0; i < TT_STAGE_COUNT; ++i) {
       ctx->stage_ms[i] = -1.f;
@@ -875,7 +950,7 @@ tt_status tt_sync(tt_ctx* ctx, tt_result* results) {
 
 tt_status tt_debug_tensor(tt_ctx* ctx, tt_state* st, int32_t which, float* host_dst, size_t cap) {
   if (!ctx || !owns_state(ctx, st) || !host_dst) return ctx ? fail(ctx, TT_ERR_INVALID_ARG, "bad state or null buffer") : TT_ERR_INVALID_ARG;
-  if (ctx->in_flight) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
+  if (ctx->q_count) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
   TT_CUDA(ctx, cudaSetDevice(ctx->dev));
   const int plane = ctx->Hm * ctx->Wm;
   const int pos = st->last_pos;
@@ -889,7 +964,8 @@ tt_status tt_debug_tensor(tt_ctx* ctx, tt_state* st, int32_t which, float* host_
     tt_status r = which == TT_TENSOR_H ? tt_state_export(ctx, st, host_dst, other.data()) : tt_state_export(ctx, st, other.data(), host_dst);
     return r;
   }
-  if (pos < 0) return fail(ctx, TT_ERR_NOT_READY, "this state was not part of the last submit");
+  if (pos < 0 || ctx->last_done < 0) return fail(ctx, TT_ERR_NOT_READY, "this state was not part of the last submit");
+  bind_slot(ctx, ctx->last_done);
   if (which == TT_TENSOR_PRE) {
     n = (size_t)3 * ctx->cfg.net_h * ctx->cfg.net_w;
     src = ctx->pre + (size_t)pos * n;
@@ -917,7 +993,7 @@ tt_status tt_debug_tensor(tt_ctx* ctx, tt_state* st, int32_t which, float* host_
 
 tt_status tt_set_profiling(tt_ctx* ctx, int32_t on) {
   if (!ctx) return TT_ERR_INVALID_ARG;
-  if (ctx->in_flight) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
+  if (ctx->q_count) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
   ctx->profiling = on != 0;
   ctx->stage_valid = false;
   return TT_OK;
@@ -925,7 +1001,6 @@ tt_status tt_set_profiling(tt_ctx* ctx, int32_t on) {
 
 tt_status tt_get_stage_times(tt_ctx* ctx, float* ms) {
   if (!ctx || !ms) return TT_ERR_INVALID_ARG;
-  if (ctx->in_flight) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
   for (int i = 0; i < TT_STAGE_COUNT; ++i) ms[i] = ctx->stage_valid ? ctx->stage_ms[i] : -1.f;
   return TT_OK;
 }

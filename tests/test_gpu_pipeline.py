@@ -259,6 +259,43 @@ def test_runs_are_bitwise_reproducible(cuda_device):
         assert np.array_equal(outs[0][1][k], outs[1][1][k]) and np.array_equal(outs[0][2][k], outs[1][2][k])
 
 
+def test_two_submits_in_flight_match_serial_execution(cuda_device):
+    """Software-pipelined use (submit t+1 before sync t, pinned host frames over the copy stream) must give
+    bit for bit what one-at-a-time execution gives, with results returned oldest first."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="pipe", src_w=214, src_h=120, net_w=160, net_h=120, overlay=True)
+    K, n = 2, 6
+    frames = [[torch.from_numpy(f).pin_memory() for f in fs] for fs in _frames(wl, K, n)]
+
+    def collect(ctx, r):
+        return [(x["frame_index"], ctx.fetch_probs(x), ctx.fetch_overlay(x), x["conf"].copy(), x["count"].copy()) for x in r]
+
+    ctx, states, _ = _make(wl, K, overlay=True)
+    serial = []
+    for t in range(n):
+        ctx.submit_frames([frames[k][t] for k in range(K)], states, frame_index=t)
+        serial.append(collect(ctx, ctx.sync()))
+    h_serial = [ctx.state_export(s) for s in states]
+    ctx.destroy()
+
+    ctx, states, _ = _make(wl, K, overlay=True)
+    piped = []
+    ctx.submit_frames([frames[k][0] for k in range(K)], states, frame_index=0)
+    for t in range(1, n):
+        ctx.submit_frames([frames[k][t] for k in range(K)], states, frame_index=t)
+        piped.append(collect(ctx, ctx.sync()))          # results of tick t-1 while tick t is in flight
+    piped.append(collect(ctx, ctx.sync()))
+    h_piped = [ctx.state_export(s) for s in states]
+    ctx.destroy()
+    for t in range(n):
+        for k in range(K):
+            a, b = serial[t][k], piped[t][k]
+            assert a[0] == b[0] == t
+            assert np.array_equal(a[1], b[1]) and np.array_equal(a[2], b[2])
+            assert np.array_equal(a[3], b[3]) and np.array_equal(a[4], b[4])
+    for k in range(K):
+        assert np.array_equal(h_serial[k][0], h_piped[k][0]) and np.array_equal(h_serial[k][1], h_piped[k][1])
+
+
 def test_boundary_error_paths(cuda_device):
     wl = tt_synth.workload("cfg0")
     ctx, (st, st2), w = _make(wl, K=2)
@@ -279,12 +316,17 @@ def test_boundary_error_paths(cuda_device):
         ctx.submit_frames([], [])
     assert e.value.status == 1
     ctx.submit_frames([f], [st])
+    ctx.submit_frames([f], [st2])                               # a second submit may be in flight
     with pytest.raises(binding.TTError) as e:
-        ctx.submit_frames([f], [st2])
-    assert e.value.status == 6                                  # one submit in flight
+        ctx.submit_frames([f], [st])
+    assert e.value.status == 6                                  # but not a third
     with pytest.raises(binding.TTError) as e:
         ctx.state_reset(st)
     assert e.value.status == 6
+    assert len(ctx.sync()) == 1
+    with pytest.raises(binding.TTError) as e:
+        ctx.state_export(st)
+    assert e.value.status == 6                                  # still one in flight
     assert len(ctx.sync()) == 1
     other, (so,), _ = _make(wl)
     with pytest.raises(binding.TTError) as e:
