@@ -246,7 +246,8 @@ tt_status tt_preprocess(const uint8_t* src_dev, int32_t K, int64_t src_frame_str
  * for TT_CONF_GAP_LINEAR) are device fp32 [n_tools][hidden] / [n_tools].
  * Outputs (device): logits, probs fp32 [K][n_tools][Hm][Wm]; masks uint8 same shape;
  * results: K tt_result records of which conf, cx, cy, count are written.
- * scratch_dev: tt_postprocess_scratch_bytes(...) bytes of device memory, contents ignored.
+ * scratch_dev: tt_postprocess_scratch_bytes(...) bytes of device memory, 8-byte aligned; the call
+ * clears it first, contents on entry are ignored.
  * hidden must be a multiple of 4 and at most 512.
  */
 size_t tt_postprocess_scratch_bytes(int32_t K, int32_t hm, int32_t wm, int32_t hidden, int32_t n_tools);
@@ -271,16 +272,17 @@ tt_status tt_postprocess(const float* h_dev, int32_t channels_last, int32_t K, i
  * Limits and rules:
  *   - tt_postprocess_scratch_bytes(K, hm, wm, hidden, n_tools) must not exceed
  *     TT_POSTPROCESS_STATIC_SCRATCH_BYTES, else TT_ERR_UNSUPPORTED is returned and nothing runs
- *     (4 MiB covers 8 streams of a 160x90 grid with 256 hidden channels);
+ *     (32 KiB: 8 streams with up to 468 hidden channels, any grid size; 8 streams of 512 hidden
+ *     channels need 35 KB and are refused, 7 such streams fit);
  *   - the first call on a device looks up the array's device address (with that device
  *     current); make that first call before starting any stream capture;
- *   - all calls on a device share the one array.  It keeps whatever the previous call left;
- *     every value that is read is written first within the same call, so nothing needs to be
- *     cleared, but two calls whose kernels overlap on the GPU (different streams without an
- *     ordering between them) race on it.  Serialise them.
+ *   - all calls on a device share the one array.  It keeps whatever the previous call left; the
+ *     accumulators in it must start at zero, so every call clears the part it uses (a memset on
+ *     `cuda_stream`) before its kernel runs.  Two calls whose kernels overlap on the GPU
+ *     (different streams without an ordering between them) race on the array.  Serialise them.
  * Everything else (arguments, layouts, outputs, errors) is as for tt_postprocess.
  */
-#define TT_POSTPROCESS_STATIC_SCRATCH_BYTES (4u << 20)
+#define TT_POSTPROCESS_STATIC_SCRATCH_BYTES (32u << 10)
 tt_status tt_postprocess_static(const float* h_dev, int32_t channels_last, int32_t K, int32_t hm, int32_t wm,
                                 int32_t hidden, int32_t n_tools, const float* head_w_dev, const float* head_b_dev,
                                 const float* conf_w_dev, const float* conf_b_dev, int32_t conf_mode, float threshold,

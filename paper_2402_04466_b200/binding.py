@@ -30,7 +30,7 @@ EXPORTED_SYMBOLS = [
     "tt_set_profiling", "tt_get_stage_times", "tt_get_counters",
     "tt_preprocess", "tt_postprocess_scratch_bytes", "tt_postprocess", "tt_postprocess_static", "tt_overlay",
 ]
-TT_POSTPROCESS_STATIC_SCRATCH_BYTES = 4 << 20
+TT_POSTPROCESS_STATIC_SCRATCH_BYTES = 32 << 10
 STAGE_NAMES = ["h2d", "preprocess", "enc0", "enc1", "enc2", "enc3", "convlstm", "postprocess", "overlay"]
 
 

@@ -1,12 +1,12 @@
 // S4 + S5: mask head (1x1 conv hidden -> tools), sigmoid, threshold, per-tool confidence
 // and mask centroid.  HBM-bound: the hidden state is read exactly once.
 //
-// Pass 1 (post_tile_kernel): a block stages 64 pixels x Ch hidden values in shared memory
-// with coalesced 128-bit loads, four threads per pixel form the T dot products, the masks,
-// logits and probabilities are written, and the block's partial sums (count, sum x, sum y
-// as integers; sum p and per-channel sum h as floats) are written to scratch.
-// Pass 2 (post_finalize_kernel): one block per stream adds the partials in a fixed order
-// (bitwise reproducible, no float atomics) and forms confidence and centroid.
+// Generic kernel (post_tile_kernel): a block stages 64 pixels x Ch hidden values in shared
+// memory with coalesced 128-bit loads, four threads per pixel form the T dot products, and the
+// masks, logits and probabilities are written.
+// The block's partial sums go into per-stream accumulators with integer atomics (fixed point for
+// the float sums: bitwise reproducible whatever the order); the block that finishes a stream last
+// forms confidence and centroid and re-zeroes the accumulators.
 #include <mutex>
 
 #include "tt_internal.h"
@@ -20,21 +20,78 @@ constexpr int ROW_PAD = 16;    // floats of padding per staged pixel row
 
 __host__ __device__ inline int post_blocks_per_img(int plane) { return (plane + PIX - 1) / PIX; }
 
+// Scratch: per-stream accumulators that the tile blocks add into with integer atomics (the order
+// of integer additions does not matter, so results stay bitwise reproducible).  Floating-point
+// sums (probabilities, pooled hidden state) are accumulated in fixed point with 30 fractional
+// bits.  The block that finishes a stream last turns the accumulators into the result record and
+// zeroes them again, so the scratch must be zero before a launch and is zero after it.
+constexpr float FIX_SCALE = 1073741824.0f;          // 2^30
+constexpr float FIX_INV = 1.0f / 1073741824.0f;
+
 struct ScratchLayout {
-  size_t off_int, off_p, off_h, total;
+  size_t off_counter, off_acc, acc_stride, total;   // acc block per stream: [Ch] pooled sums, then [TT_MAX_TOOLS][4]
 };
 __host__ __device__ inline ScratchLayout scratch_layout(int K, int plane, int ch, int T) {
-  const size_t nb = (size_t)K * post_blocks_per_img(plane);
+  (void)plane; (void)T;
   ScratchLayout l;
-  l.off_int = 0;
-  l.off_p = l.off_int + nb * TT_MAX_TOOLS * 4 * sizeof(int32_t);
-  l.off_h = l.off_p + nb * TT_MAX_TOOLS * sizeof(float);
-  l.total = l.off_h + nb * (size_t)ch * sizeof(float);
+  l.off_counter = 0;
+  l.off_acc = 256;                                   // TT_MAX_STREAMS counters fit in front
+  l.acc_stride = ((size_t)ch + TT_MAX_TOOLS * 4) * sizeof(long long);
+  l.total = l.off_acc + (size_t)K * l.acc_stride;
   l.total = (l.total + 255) & ~(size_t)255;
   return l;
 }
 
+__device__ __forceinline__ long long to_fixed(float v) { return __float2ll_rn(v * FIX_SCALE); }
+
 __device__ __forceinline__ float sigmoid_acc(float z) { return 1.0f / (1.0f + expf(-z)); }
+
+// Called by every thread of a tile block after the block has added its partial sums into the
+// stream's accumulators.  The last block of the stream to arrive finalises: confidence, count,
+// centroid -> result record; accumulators and counter back to zero.
+__device__ __forceinline__ void finish_stream(const PostParams& p, int n, int nb, int tid) {
+  __shared__ float s_gap_fin[512];
+  __shared__ int s_last;
+  const int plane = p.Hm * p.Wm, Ch = p.Ch, T = p.T;
+  const ScratchLayout sl = scratch_layout(p.K, plane, Ch, T);
+  uint8_t* scr = reinterpret_cast<uint8_t*>(p.scratch);
+  unsigned int* counter = reinterpret_cast<unsigned int*>(scr + sl.off_counter) + n;
+  long long* acc = reinterpret_cast<long long*>(scr + sl.off_acc + (size_t)n * sl.acc_stride);
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(counter, 1u) == (unsigned int)(nb - 1));
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const float inv_plane = 1.0f / (float)plane;
+  if (p.conf_mode == TT_CONF_GAP_LINEAR) {
+    for (int c = tid; c < Ch; c += POST_THREADS) s_gap_fin[c] = (float)((double)__ldcg(acc + c) * (double)FIX_INV) * inv_plane;
+  }
+  __syncthreads();
+  const int warp = tid >> 5, lane = tid & 31;
+  if (warp < T) {
+    const int t = warp;
+    float a = 0.0f;
+    if (p.conf_mode == TT_CONF_GAP_LINEAR)
+      for (int c = lane; c < Ch; c += 32) a = fmaf(__ldg(p.conf_w + t * Ch + c), s_gap_fin[c], a);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
+    if (lane == 0) {
+      const long long* st = acc + Ch + t * 4;
+      const long long cnt = __ldcg(st + 0), sx = __ldcg(st + 1), sy = __ldcg(st + 2), spf = __ldcg(st + 3);
+      const float conf = p.conf_mode == TT_CONF_GAP_LINEAR ? sigmoid_acc(a + __ldg(p.conf_b + t))
+                                                          : (float)((double)spf * (double)FIX_INV) * inv_plane;
+      tt_result* r = p.results + n;
+      r->conf[t] = conf;
+      r->count[t] = (int32_t)cnt;
+      r->cx[t] = cnt ? (float)((double)sx / (double)cnt) : -1.0f;
+      r->cy[t] = cnt ? (float)((double)sy / (double)cnt) : -1.0f;
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < Ch + TT_MAX_TOOLS * 4; i += POST_THREADS) acc[i] = 0;
+  if (tid == 0) *counter = 0u;
+}
 
 __global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const __grid_constant__ PostParams p) {
   extern __shared__ __align__(16) float s_mem[];
@@ -145,10 +202,7 @@ __global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const __grid_co
   __syncthreads();
 
   const ScratchLayout sl = scratch_layout(p.K, plane, Ch, T);
-  uint8_t* scr = reinterpret_cast<uint8_t*>(p.scratch);
-  int32_t* part_i = reinterpret_cast<int32_t*>(scr + sl.off_int) + (size_t)blockIdx.x * TT_MAX_TOOLS * 4;
-  float* part_p = reinterpret_cast<float*>(scr + sl.off_p) + (size_t)blockIdx.x * TT_MAX_TOOLS;
-  float* part_h = reinterpret_cast<float*>(scr + sl.off_h) + (size_t)blockIdx.x * Ch;
+  long long* sacc = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(p.scratch) + sl.off_acc + (size_t)n * sl.acc_stride);
   if (tid < T) {
     int cnt = 0, sx = 0, sy = 0;
     float sp = 0.0f;
@@ -158,19 +212,20 @@ __global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const __grid_co
       sy += s_red_i[(w * TT_MAX_TOOLS + tid) * 3 + 2];
       sp += s_red_f[w * TT_MAX_TOOLS + tid];
     }
-    part_i[tid * 4 + 0] = cnt;
-    part_i[tid * 4 + 1] = sx;
-    part_i[tid * 4 + 2] = sy;
-    part_i[tid * 4 + 3] = 0;
-    part_p[tid] = sp;
+    unsigned long long* st = reinterpret_cast<unsigned long long*>(sacc + Ch + tid * 4);
+    atomicAdd(st + 0, (unsigned long long)(long long)cnt);
+    atomicAdd(st + 1, (unsigned long long)(long long)sx);
+    atomicAdd(st + 2, (unsigned long long)(long long)sy);
+    atomicAdd(st + 3, (unsigned long long)to_fixed(sp));
   }
   if (p.conf_mode == TT_CONF_GAP_LINEAR) {
     for (int c = tid; c < Ch; c += POST_THREADS) {
       float s = 0.0f;
       for (int i = 0; i < npix; ++i) s += s_tile[i * row + c];
-      part_h[c] = s;
+      atomicAdd(reinterpret_cast<unsigned long long*>(sacc + c), (unsigned long long)to_fixed(s));
     }
   }
+  finish_stream(p, n, nb, tid);
 }
 
 // Channels-last fast path (hidden a multiple of 128): no shared-memory staging of the hidden
@@ -319,10 +374,7 @@ __global__ void __launch_bounds__(POST_THREADS) post_direct_kernel(const __grid_
   __syncthreads();
 
   const ScratchLayout sl = scratch_layout(p.K, plane, CH, T);
-  uint8_t* scr = reinterpret_cast<uint8_t*>(p.scratch);
-  int32_t* part_i = reinterpret_cast<int32_t*>(scr + sl.off_int) + (size_t)blockIdx.x * TT_MAX_TOOLS * 4;
-  float* part_p = reinterpret_cast<float*>(scr + sl.off_p) + (size_t)blockIdx.x * TT_MAX_TOOLS;
-  float* part_h = reinterpret_cast<float*>(scr + sl.off_h) + (size_t)blockIdx.x * CH;
+  long long* sacc = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(p.scratch) + sl.off_acc + (size_t)n * sl.acc_stride);
   if (tid < T) {
     int c = 0, x = 0, y = 0;
     float f = 0.0f;
@@ -332,89 +384,21 @@ __global__ void __launch_bounds__(POST_THREADS) post_direct_kernel(const __grid_
       y += s_red_i[(w * TT_MAX_TOOLS + tid) * 3 + 2];
       f += s_red_f[w * TT_MAX_TOOLS + tid];
     }
-    part_i[tid * 4 + 0] = c;
-    part_i[tid * 4 + 1] = x;
-    part_i[tid * 4 + 2] = y;
-    part_i[tid * 4 + 3] = 0;
-    part_p[tid] = f;
+    unsigned long long* st = reinterpret_cast<unsigned long long*>(sacc + CH + tid * 4);
+    atomicAdd(st + 0, (unsigned long long)(long long)c);
+    atomicAdd(st + 1, (unsigned long long)(long long)x);
+    atomicAdd(st + 2, (unsigned long long)(long long)y);
+    atomicAdd(st + 3, (unsigned long long)to_fixed(f));
   }
   if (p.conf_mode == TT_CONF_GAP_LINEAR) {
     for (int c = tid; c < CH; c += POST_THREADS) {
       float a = 0.0f;
 #pragma unroll
       for (int w = 0; w < 8; ++w) a += s_gapw[w][c];
-      part_h[c] = a;
+      atomicAdd(reinterpret_cast<unsigned long long*>(sacc + c), (unsigned long long)to_fixed(a));
     }
   }
-}
-
-// One block of 1024 threads per stream.  Pooled hidden state: the tile blocks are split into
-// G = 1024 / Ch interleaved groups, thread (g, c) adds channel c over group g's blocks in
-// order, and the G group sums are added in order.  Tool statistics: warp t reduces the partials
-// of tool t (lanes stride over the tile blocks, then a fixed shuffle tree).  The order of the
-// additions never depends on timing, so results are bitwise reproducible.
-constexpr int FIN_THREADS = 1024;
-
-__global__ void __launch_bounds__(FIN_THREADS) post_finalize_kernel(const __grid_constant__ PostParams p) {
-  __shared__ float s_part[FIN_THREADS];
-  __shared__ float s_gap[512];
-  const int n = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int plane = p.Hm * p.Wm, Ch = p.Ch, T = p.T;
-  const int nb = post_blocks_per_img(plane);
-  const ScratchLayout sl = scratch_layout(p.K, plane, Ch, T);
-  const uint8_t* scr = reinterpret_cast<const uint8_t*>(p.scratch);
-  const int4* part_i = reinterpret_cast<const int4*>(scr + sl.off_int) + (size_t)n * nb * TT_MAX_TOOLS;
-  const float* part_p = reinterpret_cast<const float*>(scr + sl.off_p) + (size_t)n * nb * TT_MAX_TOOLS;
-  const float* part_h = reinterpret_cast<const float*>(scr + sl.off_h) + (size_t)n * nb * Ch;
-  const float inv_plane = 1.0f / (float)plane;
-
-  if (p.conf_mode == TT_CONF_GAP_LINEAR) {
-    const int G = FIN_THREADS / Ch;          // Ch <= 512, so G >= 2
-    const int g = tid / Ch, c = tid - g * Ch;
-    float s = 0.0f;
-    if (g < G) {
-#pragma unroll 32
-      for (int b = g; b < nb; b += G) s += part_h[(size_t)b * Ch + c];
-    }
-    s_part[tid] = s;
-    __syncthreads();
-    if (tid < Ch) {
-      float a = 0.0f;
-      for (int k = 0; k < G; ++k) a += s_part[k * Ch + tid];
-      s_gap[tid] = a * inv_plane;
-    }
-  }
-  __syncthreads();
-  if (warp < T) {
-    const int t = warp;
-    long long cnt = 0, sx = 0, sy = 0;
-    float sp = 0.0f;
-#pragma unroll 8
-    for (int b = lane; b < nb; b += 32) {
-      const int4 v = part_i[(size_t)b * TT_MAX_TOOLS + t];
-      cnt += v.x; sx += v.y; sy += v.z;
-      sp += part_p[(size_t)b * TT_MAX_TOOLS + t];
-    }
-    float a = 0.0f;
-    if (p.conf_mode == TT_CONF_GAP_LINEAR)
-      for (int c = lane; c < Ch; c += 32) a = fmaf(__ldg(p.conf_w + t * Ch + c), s_gap[c], a);
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-      cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
-      sx += __shfl_xor_sync(0xffffffffu, sx, d);
-      sy += __shfl_xor_sync(0xffffffffu, sy, d);
-      sp += __shfl_xor_sync(0xffffffffu, sp, d);
-      a += __shfl_xor_sync(0xffffffffu, a, d);
-    }
-    if (lane == 0) {
-      const float conf = p.conf_mode == TT_CONF_GAP_LINEAR ? sigmoid_acc(a + __ldg(p.conf_b + t)) : sp * inv_plane;
-      tt_result* r = p.results + n;
-      r->conf[t] = conf;
-      r->count[t] = (int32_t)cnt;
-      r->cx[t] = cnt ? (float)((double)sx / (double)cnt) : -1.0f;
-      r->cy[t] = cnt ? (float)((double)sy / (double)cnt) : -1.0f;
-    }
-  }
+  finish_stream(p, n, nb, tid);
 }
 
 // Scratch of the entry point that allocates nothing: one fixed array inside the library image.
@@ -472,9 +456,6 @@ cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s) {
   else if (direct && p.Ch == 256) post_direct_kernel<2><<<p.K * nb, POST_THREADS, dsm, s>>>(p);
   else if (direct) post_direct_kernel<4><<<p.K * nb, POST_THREADS, dsm, s>>>(p);
   else post_tile_kernel<<<p.K * nb, POST_THREADS, post_smem_bytes(p.Ch), s>>>(p);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  post_finalize_kernel<<<p.K, FIN_THREADS, 0, s>>>(p);
   return cudaGetLastError();
 }
 

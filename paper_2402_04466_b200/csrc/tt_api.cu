@@ -943,6 +943,8 @@ tt_status tt_sync(tt_ctx* ctx, tt_result* results) {
     const int code = *ctx->status_host;
     *ctx->status_host = 0;
     cudaMemsetAsync(ctx->status_dev, 0, sizeof(int32_t), ctx->stream);
+    // a tick that gave up may have left partial sums in the post-processing accumulators
+    cudaMemsetAsync(ctx->post_scratch, 0, post_scratch_bytes(ctx->cfg.max_streams, ctx->Hm, ctx->Wm, ctx->Ch, ctx->T), ctx->stream);
     return fail(ctx, TT_ERR_DEVICE_STATUS, "a kernel gave up a bounded wait (code 0x%x); results of this tick are invalid", code);
   }
   return TT_OK;
@@ -1054,6 +1056,8 @@ tt_status tt_postprocess(const float* h_dev, int32_t channels_last, int32_t K, i
   p.zthr = (float)std::log((double)threshold / (1.0 - (double)threshold));
   p.logits = logits_dev; p.probs = probs_dev; p.masks = masks_dev; p.bits = nullptr; p.results = results_dev;
   p.scratch = scratch_dev;
+  e = cudaMemsetAsync(scratch_dev, 0, post_scratch_bytes(K, hm, wm, hidden, n_tools), reinterpret_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return fail(nullptr, TT_ERR_CUDA, "tt_postprocess: %s", cudaGetErrorString(e));
   e = launch_postprocess(p, reinterpret_cast<cudaStream_t>(cuda_stream));
   if (e != cudaSuccess) return fail(nullptr, TT_ERR_CUDA, "tt_postprocess: %s", cudaGetErrorString(e));
   return TT_OK;
@@ -1092,6 +1096,9 @@ tt_status tt_postprocess_static(const float* h_dev, int32_t channels_last, int32
   p.zthr = (float)std::log((double)threshold / (1.0 - (double)threshold));
   p.logits = logits_dev; p.probs = probs_dev; p.masks = masks_dev; p.bits = nullptr; p.results = results_dev;
   p.scratch = scratch;
+  // the accumulators in the shared array must start at zero, whatever an earlier call left there
+  e = cudaMemsetAsync(scratch, 0, need, reinterpret_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return fail(nullptr, TT_ERR_CUDA, "tt_postprocess_static: %s", cudaGetErrorString(e));
   e = launch_postprocess(p, reinterpret_cast<cudaStream_t>(cuda_stream));
   if (e != cudaSuccess) return fail(nullptr, TT_ERR_CUDA, "tt_postprocess_static: %s", cudaGetErrorString(e));
   return TT_OK;

@@ -54,9 +54,9 @@ def test_static_scratch_matches_caller_scratch_twice_in_a_row(cuda_device):
 
 def test_static_scratch_rejects_problems_beyond_its_size(cuda_device):
     lib = binding.load_library()
-    assert lib.tt_postprocess_scratch_bytes(8, 512, 512, 512, 8) > binding.TT_POSTPROCESS_STATIC_SCRATCH_BYTES
+    assert lib.tt_postprocess_scratch_bytes(8, 16, 16, 512, 8) > binding.TT_POSTPROCESS_STATIC_SCRATCH_BYTES
     d = torch.zeros(64, dtype=torch.float32, device=cuda_device)      # never touched: the call is refused up front
-    st = lib.tt_postprocess_static(d.data_ptr(), 1, 8, 512, 512, 512, 8, d.data_ptr(), d.data_ptr(), None, None, 0, 0.5,
+    st = lib.tt_postprocess_static(d.data_ptr(), 1, 8, 16, 16, 512, 8, d.data_ptr(), d.data_ptr(), None, None, 0, 0.5,
                                    d.data_ptr(), d.data_ptr(), d.data_ptr(), d.data_ptr(), None)
     assert st == 2
     assert b"scratch" in lib.tt_last_error(None)
