@@ -198,6 +198,57 @@ tt_status tt_sync(tt_ctx* ctx, tt_result* results);
 tt_status tt_debug_tensor(tt_ctx* ctx, tt_state* st, int32_t which, float* host_dst, size_t cap);
 
 /*
+ * tt_query — non-blocking: TT_OK when the oldest submit in flight has finished (tt_sync will not
+ * block), TT_ERR_NOT_READY when it is still running or nothing is in flight.
+ */
+tt_status tt_query(tt_ctx* ctx);
+
+/*
+ * Batch planner for unsynchronised arrivals (host logic only, no CUDA calls, no context needed).
+ * The paper's N applications run unsynchronised (Section V-B) and are protected from each other
+ * by an admission control that refuses a client the GPU cannot accommodate (Section IV-A,
+ * "Admission Control").  With one shared launch sequence the same questions become: which
+ * waiting frames go into the next tick, and may another stream join?
+ *   - tt_sched_admit: a new stream is refused (TT_ERR_ADMISSION) when all max_streams slots are
+ *     taken or when the predicted tick time with one more stream exceeds budget_fraction *
+ *     deadline_ns.  The prediction is tick_ms_base + tick_ms_per_stream * K until ticks of that
+ *     size have been observed, then an exponential average of the observed times.
+ *   - tt_sched_arrive: a frame of an admitted stream arrived at t_ns (caller's monotonic clock).
+ *     If the stream's previous frame is still waiting the new frame is dropped: TT_ERR_ADMISSION.
+ *   - tt_sched_next: at time now_ns, returns in K / stream_ids / frame_indices / arrival_ns
+ *     (arrays of max_streams entries) the batch to launch now, or K = 0 and in *wake_ns the time
+ *     to ask again (UINT64_MAX: nothing waiting, or max_in_flight batches already launched — ask
+ *     again after a completion).  With nothing in flight a waiting frame is released at once.
+ *     While a batch is in flight, frames are held to coalesce and released as soon as every
+ *     admitted stream has a frame waiting, or the oldest waiting frame has waited window_ns, or
+ *     waiting longer would push the oldest frame past budget_fraction * deadline_ns given the
+ *     predicted tick time.
+ *   - tt_sched_complete: the oldest launched batch finished (device time gpu_ms, at done_ns);
+ *     updates the cost model and counts frames that finished later than arrival + deadline_ns.
+ */
+typedef struct tt_sched tt_sched;
+typedef struct {
+  uint32_t struct_size;       /* = sizeof(tt_sched_config) */
+  int32_t max_streams;        /* 1..TT_MAX_STREAMS */
+  int32_t max_in_flight;      /* 1 or 2 batches launched and not yet completed */
+  float budget_fraction;      /* share of deadline_ns one tick may take, in (0, 1] */
+  uint64_t window_ns;         /* coalescing window */
+  uint64_t deadline_ns;       /* per-frame latency budget, e.g. 16 666 667 */
+  float tick_ms_base;         /* prior of the tick-time model */
+  float tick_ms_per_stream;
+} tt_sched_config;
+tt_status tt_sched_create(const tt_sched_config* cfg, tt_sched** out);
+tt_status tt_sched_destroy(tt_sched* s);
+tt_status tt_sched_admit(tt_sched* s, int32_t* stream_id);
+tt_status tt_sched_release(tt_sched* s, int32_t stream_id);
+tt_status tt_sched_arrive(tt_sched* s, int32_t stream_id, uint64_t frame_index, uint64_t t_ns);
+tt_status tt_sched_next(tt_sched* s, uint64_t now_ns, int32_t* K, int32_t* stream_ids, uint64_t* frame_indices,
+                        uint64_t* arrival_ns, uint64_t* wake_ns);
+tt_status tt_sched_complete(tt_sched* s, float gpu_ms, uint64_t done_ns);
+tt_status tt_sched_predict_ms(const tt_sched* s, int32_t K, float* ms);
+tt_status tt_sched_stats(const tt_sched* s, uint64_t* batches, uint64_t* frames, uint64_t* dropped, uint64_t* missed);
+
+/*
  * Measurement hooks (the paper times every operator's input and output, Section II-C, data
  * flow tracking; here CUDA events on the context's stream bracket each stage of a tick).
  * tt_set_profiling(on != 0) makes every following submit record stage events.

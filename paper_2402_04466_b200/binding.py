@@ -27,7 +27,9 @@ TENSOR_IDS = {"pre": 0, "enc0": 1, "enc1": 2, "enc2": 3, "enc3": 4, "h": 8, "c":
 EXPORTED_SYMBOLS = [
     "tt_abi_version", "tt_create", "tt_destroy", "tt_last_error", "tt_map_size", "tt_state_create",
     "tt_state_reset", "tt_state_export", "tt_state_import", "tt_submit_frames", "tt_sync", "tt_debug_tensor",
-    "tt_set_profiling", "tt_get_stage_times", "tt_get_counters",
+    "tt_set_profiling", "tt_get_stage_times", "tt_get_counters", "tt_query",
+    "tt_sched_create", "tt_sched_destroy", "tt_sched_admit", "tt_sched_release", "tt_sched_arrive", "tt_sched_next",
+    "tt_sched_complete", "tt_sched_predict_ms", "tt_sched_stats",
     "tt_preprocess", "tt_postprocess_scratch_bytes", "tt_postprocess", "tt_postprocess_static", "tt_overlay",
 ]
 TT_POSTPROCESS_STATIC_SCRATCH_BYTES = 32 << 10
@@ -76,6 +78,12 @@ class tt_result(C.Structure):
                 ("gpu_ms", C.c_float), ("reserved_", C.c_int32)]
 
 
+class tt_sched_config(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("max_streams", C.c_int32), ("max_in_flight", C.c_int32),
+                ("budget_fraction", C.c_float), ("window_ns", C.c_uint64), ("deadline_ns", C.c_uint64),
+                ("tick_ms_base", C.c_float), ("tick_ms_per_stream", C.c_float)]
+
+
 _LIB = None
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtt.so")
 
@@ -109,6 +117,17 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.tt_set_profiling.argtypes = [vp, i32]
     lib.tt_get_stage_times.argtypes = [vp, C.POINTER(C.c_float)]
     lib.tt_get_counters.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+    lib.tt_query.argtypes = [vp]
+    u64p = C.POINTER(C.c_uint64)
+    lib.tt_sched_create.argtypes = [C.POINTER(tt_sched_config), C.POINTER(vp)]
+    lib.tt_sched_destroy.argtypes = [vp]
+    lib.tt_sched_admit.argtypes = [vp, C.POINTER(i32)]
+    lib.tt_sched_release.argtypes = [vp, i32]
+    lib.tt_sched_arrive.argtypes = [vp, i32, C.c_uint64, C.c_uint64]
+    lib.tt_sched_next.argtypes = [vp, C.c_uint64, C.POINTER(i32), C.POINTER(i32), u64p, u64p, u64p]
+    lib.tt_sched_complete.argtypes = [vp, f32, C.c_uint64]
+    lib.tt_sched_predict_ms.argtypes = [vp, i32, C.POINTER(f32)]
+    lib.tt_sched_stats.argtypes = [vp, u64p, u64p, u64p, u64p]
     lib.tt_preprocess.argtypes = [vp, i32, i64, i32, i32, i32, vp, i32, i32, f32, f32, f32, vp]
     lib.tt_postprocess_scratch_bytes.argtypes = [i32, i32, i32, i32, i32]
     lib.tt_postprocess_scratch_bytes.restype = C.c_size_t
@@ -284,6 +303,10 @@ class Context:
         _check(self.lib, self.lib.tt_get_counters(self.handle, C.byref(a), C.byref(b)), self.handle)
         return int(a.value), int(b.value)
 
+    def query(self) -> bool:
+        """True when the oldest submit in flight has finished (tt_sync would not block)."""
+        return self.lib.tt_query(self.handle) == TT_OK
+
     def last_error(self) -> str:
         m = self.lib.tt_last_error(self.handle)
         return m.decode() if m else ""
@@ -315,6 +338,84 @@ class Context:
 
     def fetch_overlay(self, result: Dict) -> np.ndarray:
         return _copy_from_device(result["overlay_dev"], (self.cfg.src_h, self.cfg.src_w, 4), np.uint8)
+
+
+class Scheduler:
+    """tt_sched_*: batch planner for unsynchronised arrivals (host logic only, usable without a GPU)."""
+
+    NEVER = 2 ** 64 - 1
+
+    def __init__(self, max_streams: int, window_ns: int, deadline_ns: int = 16_666_667, max_in_flight: int = 2,
+                 budget_fraction: float = 0.5, tick_ms_base: float = 0.1, tick_ms_per_stream: float = 0.02):
+        self.lib = load_library()
+        cfg = tt_sched_config(C.sizeof(tt_sched_config), max_streams, max_in_flight, budget_fraction, window_ns,
+                              deadline_ns, tick_ms_base, tick_ms_per_stream)
+        h = C.c_void_p()
+        st = self.lib.tt_sched_create(C.byref(cfg), C.byref(h))
+        if st != TT_OK:
+            raise TTError(st, "tt_sched_create")
+        self.handle, self.max_streams = h, max_streams
+
+    def destroy(self):
+        if self.handle:
+            self.lib.tt_sched_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def admit(self) -> int:
+        sid = C.c_int32()
+        st = self.lib.tt_sched_admit(self.handle, C.byref(sid))
+        if st != TT_OK:
+            raise TTError(st, "stream refused by admission control")
+        return sid.value
+
+    def release(self, stream_id: int):
+        st = self.lib.tt_sched_release(self.handle, stream_id)
+        if st != TT_OK:
+            raise TTError(st, "tt_sched_release")
+
+    def arrive(self, stream_id: int, frame_index: int, t_ns: int) -> bool:
+        """False when the frame was dropped because the stream's previous frame is still waiting."""
+        st = self.lib.tt_sched_arrive(self.handle, stream_id, frame_index, t_ns)
+        if st == TT_OK:
+            return True
+        if st == 5:
+            return False
+        raise TTError(st, "tt_sched_arrive")
+
+    def next(self, now_ns: int):
+        """-> (batch, wake_ns); batch is a list of (stream_id, frame_index, arrival_ns), empty when nothing launches now."""
+        K = C.c_int32()
+        ids = (C.c_int32 * TT_MAX_STREAMS)()
+        fi = (C.c_uint64 * TT_MAX_STREAMS)()
+        ar = (C.c_uint64 * TT_MAX_STREAMS)()
+        wake = C.c_uint64()
+        st = self.lib.tt_sched_next(self.handle, now_ns, C.byref(K), ids, fi, ar, C.byref(wake))
+        if st != TT_OK:
+            raise TTError(st, "tt_sched_next")
+        return [(ids[i], fi[i], ar[i]) for i in range(K.value)], wake.value
+
+    def complete(self, gpu_ms: float, done_ns: int):
+        st = self.lib.tt_sched_complete(self.handle, gpu_ms, done_ns)
+        if st != TT_OK:
+            raise TTError(st, "tt_sched_complete")
+
+    def predict_ms(self, K: int) -> float:
+        ms = C.c_float()
+        st = self.lib.tt_sched_predict_ms(self.handle, K, C.byref(ms))
+        if st != TT_OK:
+            raise TTError(st, "tt_sched_predict_ms")
+        return ms.value
+
+    def stats(self):
+        a, b, c, d = C.c_uint64(), C.c_uint64(), C.c_uint64(), C.c_uint64()
+        self.lib.tt_sched_stats(self.handle, C.byref(a), C.byref(b), C.byref(c), C.byref(d))
+        return {"batches": a.value, "frames": b.value, "dropped": c.value, "deadline_misses": d.value}
 
 
 class _DeviceView:

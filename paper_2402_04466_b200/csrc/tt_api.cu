@@ -950,6 +950,15 @@ tt_status tt_sync(tt_ctx* ctx, tt_result* results) {
   return TT_OK;
 }
 
+tt_status tt_query(tt_ctx* ctx) {
+  if (!ctx) return TT_ERR_INVALID_ARG;
+  if (ctx->q_count == 0) return TT_ERR_NOT_READY;
+  cudaError_t e = cudaEventQuery(ctx->slots[ctx->q_head].ev_stop);
+  if (e == cudaSuccess) return TT_OK;
+  if (e == cudaErrorNotReady) return TT_ERR_NOT_READY;
+  return fail(ctx, TT_ERR_CUDA, "cudaEventQuery: %s", cudaGetErrorString(e));
+}
+
 tt_status tt_debug_tensor(tt_ctx* ctx, tt_state* st, int32_t which, float* host_dst, size_t cap) {
   if (!ctx || !owns_state(ctx, st) || !host_dst) return ctx ? fail(ctx, TT_ERR_INVALID_ARG, "bad state or null buffer") : TT_ERR_INVALID_ARG;
   if (ctx->q_count) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");

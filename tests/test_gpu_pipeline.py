@@ -339,3 +339,57 @@ def test_boundary_error_paths(cuda_device):
     with pytest.raises(binding.TTError) as e:
         binding.Context(binding.make_config(bad), tt_synth.make_weights(bad))
     assert e.value.status == 2
+
+
+def test_staggered_arrivals_through_the_planner_match_per_stream_runs(cuda_device):
+    """Unsynchronised arrivals: four streams with different phases are coalesced by the batch planner into
+    ticks of varying composition (virtual time).  Streams are independent, so every stream must see exactly
+    the results it gets when it runs alone, whatever batches it shared."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="stagger", src_w=214, src_h=120, net_w=160, net_h=120, hidden=64)
+    K, n = 4, 10
+    period, ms = 16_666_667, 1_000_000
+    frames = _frames(wl, K, n)
+    dev_frames = [[torch.from_numpy(f).to(cuda_device) for f in fs] for fs in frames]
+    sched = binding.Scheduler(max_streams=K, window_ns=2 * ms, deadline_ns=period, max_in_flight=1)
+    sids = [sched.admit() for _ in range(K)]
+    phases = [0, 100_000, 200_000, 9 * ms]                        # streams 1, 2 arrive while stream 0's tick is in flight
+    arrivals = sorted((phases[k] + t * period + (23_000 * ((t * 7 + k) % 5)), k, t) for k in range(K) for t in range(n))
+    ctx, states, _ = _make(wl, K)
+    got = {}
+    sizes = []
+    pending = list(arrivals)
+    now, done_at, done_ms = 0, None, 0.0                          # virtual clock; a tick occupies the GPU for 300 us
+    while True:
+        if done_at is not None and now >= done_at:
+            sched.complete(done_ms, done_at)
+            done_at = None
+        batch, wake = sched.next(now)
+        if batch:
+            ctx.submit_frames([dev_frames[s][fi] for s, fi, _ in batch], [states[s] for s, _, _ in batch], frame_index=batch[0][1])
+            res = ctx.sync()
+            done_at, done_ms = now + 300_000, res[0]["gpu_ms"]
+            sizes.append(len(batch))
+            for (s, fi, _), r in zip(batch, res):
+                got[(s, fi)] = (ctx.fetch_probs(r), r["conf"].copy(), r["count"].copy(), r["cx"].copy())
+            continue
+        times = [t for t in (wake if wake != binding.Scheduler.NEVER else None, pending[0][0] if pending else None, done_at) if t is not None]
+        if not times:
+            break
+        now = max(now, min(times))
+        while pending and pending[0][0] <= now:
+            _, k, t = pending.pop(0)
+            assert sched.arrive(sids[k], t, now)
+    st = sched.stats()
+    assert st["frames"] == K * n and st["dropped"] == 0 and st["deadline_misses"] == 0
+    assert len(got) == K * n and min(sizes) == 1 and max(sizes) >= 2 and st["batches"] < K * n
+    ctx.destroy()
+    ctx1, (s1,), _ = _make(wl, 1)
+    for k in range(K):
+        ctx1.state_reset(s1)
+        for t in range(n):
+            ctx1.submit_frames([dev_frames[k][t]], [s1], frame_index=t)
+            (r,) = ctx1.sync()
+            p, conf, cnt, cx = got[(k, t)]
+            assert np.array_equal(ctx1.fetch_probs(r), p) and np.array_equal(r["conf"], conf)
+            assert np.array_equal(r["count"], cnt) and np.array_equal(r["cx"], cx)
+    ctx1.destroy()
