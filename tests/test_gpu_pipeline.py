@@ -158,6 +158,14 @@ def test_bf16_small_ragged_shapes_three_streams(cuda_device):
     _run_bf16(cuda_device, wl, 3, 3)
 
 
+def test_bf16_odd_extents_on_strided_layers(cuda_device):
+    """Odd widths and heights at every stride-2 layer: 150x110 -> 75x55 -> 38x28 -> 19x14 (parity views of unequal size)."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="bf16-odd", src_w=200, src_h=150, net_w=150, net_h=110,
+                                              enc_cout=(32, 64, 128), hidden=32)
+    assert wl.map_hw() == (14, 19)
+    _run_bf16(cuda_device, wl, 2, 3)
+
+
 def test_bf16_wide_channels_small_map(cuda_device):
     """The scale-sweep channel widths (64/128/256, hidden 256: N = 1024, K = 4608) on a small map."""
     wl = tt_synth.workload("cfg4-gain").with_(name="bf16-wide", src_w=160, src_h=120, net_w=136, net_h=104)
