@@ -9,12 +9,6 @@
 // with tcgen05.ld and applies bias + ReLU (encoder) or the whole ConvLSTM gate math
 // (sigmoid/tanh, c' = f*c + i*g, h' = o*tanh(c')) so gate pre-activations never reach HBM.
 //
-// Stride-1 layers with 64-channel slabs (the ConvLSTM) use "halo mode": the producer loads one
-// haloed 18 x 10 pixel patch per channel slab through a 5-D tensor map (8 channels, x, y, channel
-// group, image) that lands as eight [18][10][16-byte] planes -- the no-swizzle core-matrix layout --
-// and all nine taps are shifted descriptors into that one tile; only the weight slab is fetched
-// per tap.  This cuts the activation traffic from L2 nine-fold.
-//
 // Stride-2 layers read four "parity views" of their input (even/odd rows x even/odd
 // columns), each an ordinary tiled tensor map with doubled strides, so every tap is again
 // a dense box.
@@ -48,17 +42,6 @@ struct TcCfg {
   static constexpr int TMEM_COLS = 2 * BLOCK_N < 32 ? 32 : 2 * BLOCK_N;
   static constexpr int BAR_BYTES = 256;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024 /*alignment slack*/;
-  // halo mode (stride 1, 64-channel slabs): the activation ring holds haloed patches of
-  // 18 x 10 pixels x 64 channels as eight 8-channel planes ([chunk][y][x][16 bytes]); the weight
-  // ring holds one [BLOCK_N][64] slab per tap
-  static constexpr int HALO_W = 10, HALO_H = 18;
-  static constexpr int HALO_CHUNK_BYTES = HALO_H * HALO_W * 16;         // one 8-channel plane
-  static constexpr int HALO_A_BYTES = 8 * HALO_CHUNK_BYTES;             // 23040
-  static constexpr int HALO_A_STRIDE = (HALO_A_BYTES + 1023) / 1024 * 1024;
-  static constexpr int HALO_A_STAGES = 2;
-  static constexpr int HALO_B_RAW = (192 * 1024 - HALO_A_STAGES * HALO_A_STRIDE) / B_BYTES;
-  static constexpr int HALO_B_STAGES = HALO_B_RAW > 8 ? 8 : HALO_B_RAW;
-  static constexpr int HALO_SMEM_BYTES = HALO_B_STAGES * B_BYTES + HALO_A_STAGES * HALO_A_STRIDE + BAR_BYTES + 1024;
   static_assert((TMEM_COLS & (TMEM_COLS - 1)) == 0 && TMEM_COLS <= 512, "TMEM columns must be a power of two <= 512");
   static_assert(A_BYTES % 1024 == 0 && B_BYTES % 1024 == 0, "operand tiles must keep 1024-byte alignment");
 };
@@ -74,31 +57,22 @@ __device__ __forceinline__ float fast_sigmoid(float z) { return fmaf(0.5f, fast_
 
 
 // ------------------------------------------------------------------------------------ kernel
-template <int BLOCK_N, int SLAB_C, int EPI, bool HALO>
+template <int BLOCK_N, int SLAB_C, int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_constant__ ConvTcParams p) {
   using Cfg = TcCfg<BLOCK_N, SLAB_C>;
-  static_assert(!HALO || SLAB_C == 64, "halo mode is built for 64-channel slabs");
-  // ring depth: stages of (A + B) normally; in halo mode STAGES counts the weight ring and the
-  // activation ring has its own barriers behind it
-  constexpr int STAGES = HALO ? Cfg::HALO_B_STAGES : Cfg::STAGES;
-  constexpr int A_STAGES = HALO ? Cfg::HALO_A_STAGES : 0;
-  constexpr int PW = HALO ? 8 : PATCH_W;           // output patch: 8 x 16 in halo mode, 16 x 8 otherwise
-  constexpr int PH = HALO ? 16 : PATCH_H;
+  constexpr int STAGES = Cfg::STAGES;
   constexpr uint32_t LAYOUT = SLAB_C == 64 ? 2u : 4u;
   constexpr uint32_t SBO = 8u * SLAB_C * 2u;
   constexpr uint32_t IDESC = make_idesc(BLOCK_M, BLOCK_N);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* smem_a = smem + STAGES * Cfg::B_BYTES;              // halo mode: activation ring behind the weight ring
-  uint8_t* bar_mem = HALO ? smem_a + A_STAGES * Cfg::HALO_A_STRIDE : smem + STAGES * Cfg::STAGE_BYTES;
+  uint8_t* bar_mem = smem + STAGES * Cfg::STAGE_BYTES;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(bar_mem);   // [STAGES]
   uint64_t* empty_bar = full_bar + STAGES;                     // [STAGES]
   uint64_t* tfull_bar = empty_bar + STAGES;                    // [2]
   uint64_t* tempty_bar = tfull_bar + 2;                        // [2]
-  uint64_t* afull_bar = tempty_bar + 2;                        // [2] halo mode only
-  uint64_t* aempty_bar = afull_bar + 2;                        // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aempty_bar + 2);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -111,8 +85,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(tfull_bar + a), 1);
       mbar_init(smem_u32(tempty_bar + a), EPI_WARPS);
-      mbar_init(smem_u32(afull_bar + a), 1);
-      mbar_init(smem_u32(aempty_bar + a), 1);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -137,41 +109,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     // ------------------------------------------------------------------ TMA producer
     uint32_t stage = 0, phase = 0;
     bool ok = true;
-    if (HALO) {
-      // One haloed activation patch per 64-channel slab (x slabs, then h slabs), and for each of
-      // them the nine weight slabs of the taps.  The 5-D box (8 channels, 10 columns, 18 rows,
-      // 8 channel groups, 1 image) lands as eight [18][10][16-byte] planes: every tap of the
-      // 3x3 window is then a shifted view of the same shared-memory tile.
-      uint32_t a_stage = 0, a_phase = 0;
-      const int cin_total = slabs_per_tap * SLAB_C;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int nt = tile % p.n_tiles_n;
-        const int m = tile / p.n_tiles_n;
-        const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
-        int slab_global = 0;
-        for (int src = 0; src < p.n_src && ok; ++src) {
-          const void* map_a = &p.maps_a[src * 4];
-          const int img_idx = src == 0 ? p.img0.v[img] : p.img1.v[img];
-          for (int sl = 0; sl < p.slabs[src] && ok; ++sl, ++slab_global) {
-            ok = mbar_wait(smem_u32(aempty_bar + a_stage), a_phase ^ 1u, abort_flag, p.status, 0x900 + (int)a_stage);
-            if (!ok) break;
-            const uint32_t ab = smem_u32(afull_bar + a_stage);
-            mbar_arrive_expect_tx(ab, Cfg::HALO_A_BYTES);
-            tma_load_5d(smem_u32(smem_a + a_stage * Cfg::HALO_A_STRIDE), map_a, ab, 0, tx * PW - 1, ty * PH - 1, sl * 8, img_idx);
-            if (++a_stage == A_STAGES) { a_stage = 0; a_phase ^= 1u; }
-            for (int tap = 0; tap < 9; ++tap) {
-              ok = mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag, p.status, 0x100 + (int)stage);
-              if (!ok) break;
-              const uint32_t fb = smem_u32(full_bar + stage);
-              mbar_arrive_expect_tx(fb, Cfg::B_BYTES);
-              tma_load_2d(smem_u32(smem + stage * Cfg::B_BYTES), &p.map_b, fb, tap * cin_total + slab_global * SLAB_C, nt * BLOCK_N);
-              if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-            }
-          }
-        }
-      }
-    }
-    for (int tile = blockIdx.x; tile < total_tiles && ok && !HALO; tile += gridDim.x) {
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int nt = tile % p.n_tiles_n;
       const int m = tile / p.n_tiles_n;
       const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
@@ -210,7 +148,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     }
   } else if (warp == 1 && lane == 0) {
     // -------------------------------------------------------------------- MMA issuer
-    uint32_t stage = 0, phase = 0, acc_phase = 0, a_stage = 0, a_phase = 0;
+    uint32_t stage = 0, phase = 0, acc_phase = 0;
     int acc = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
@@ -218,38 +156,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
       if (!ok) break;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BLOCK_N);
-      if (HALO) {
-        uint32_t first = 1;
-        for (int sg = 0; sg < slabs_per_tap && ok; ++sg) {
-          ok = mbar_wait(smem_u32(afull_bar + a_stage), a_phase, abort_flag, p.status, 0xA00 + (int)a_stage);
-          if (!ok) break;
-          const uint32_t a_base = smem_u32(smem_a + a_stage * Cfg::HALO_A_STRIDE);
-          for (int tap = 0; tap < 9; ++tap) {
-            ok = mbar_wait(smem_u32(full_bar + stage), phase, abort_flag, p.status, 0x300 + (int)stage);
-            if (!ok) break;
-            tc_fence_after();
-            // output pixel (y, x) of the patch reads halo pixel (y + ky, x + kx): the operand of this
-            // tap starts (ky * 10 + kx) pixels into the plane; rows of an 8-row group are the 8
-            // pixels of one patch row (16 bytes apart), groups are 160 bytes apart (next row),
-            // the two 8-channel halves of a K step are one plane (2880 bytes) apart
-            const uint32_t a_tap = a_base + (uint32_t)(((tap / 3) * Cfg::HALO_W + (tap % 3)) * 16);
-            const uint64_t b_desc = make_smem_desc(smem_u32(smem + stage * Cfg::B_BYTES), SBO, LAYOUT);
-#pragma unroll
-            for (int k = 0; k < SLAB_C / UMMA_K; ++k) {
-              const uint64_t a_desc = make_smem_desc_lbo(a_tap + (uint32_t)(2 * k * Cfg::HALO_CHUNK_BYTES), Cfg::HALO_CHUNK_BYTES,
-                                                         Cfg::HALO_W * 16, 0);
-              umma_bf16(d_tmem, a_desc, b_desc + (uint64_t)(2 * k), IDESC, first ? 0u : 1u);
-              first = 0;
-            }
-            umma_commit(smem_u32(empty_bar + stage));
-            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-          }
-          if (!ok) break;
-          umma_commit(smem_u32(aempty_bar + a_stage));  // the patch is free once all nine taps have read it
-          if (++a_stage == A_STAGES) { a_stage = 0; a_phase ^= 1u; }
-        }
-      }
-      for (int it = 0; it < k_iters && !HALO; ++it) {
+      for (int it = 0; it < k_iters; ++it) {
         ok = mbar_wait(smem_u32(full_bar + stage), phase, abort_flag, p.status, 0x300 + (int)stage);
         if (!ok) break;
         tc_fence_after();
@@ -276,7 +183,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
     const int half = (warp - 2) >> 2;             // which half of the tile's columns
     const int row = quarter * 32 + lane;          // row of the 128-row tile = pixel of the patch
-    const int py = row / PW, px = row % PW;
+    const int py = row / PATCH_W, px = row % PATCH_W;
     uint32_t acc_phase = 0;
     int acc = 0;
     bool ok = true;
@@ -284,7 +191,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
       const int nt = tile % p.n_tiles_n;
       const int m = tile / p.n_tiles_n;
       const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
-      const int x = tx * PW + px, y = ty * PH + py;
+      const int x = tx * PATCH_W + px, y = ty * PATCH_H + py;
       const bool valid = x < p.Wo && y < p.Ho;
       const size_t pix = (size_t)y * p.Wo + x;
       const int col0 = nt * BLOCK_N + half * HALF_N;  // first packed output column of this warp
@@ -386,35 +293,27 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
   }
 }
 
-template <int BLOCK_N, int SLAB_C, int EPI, bool HALO>
+template <int BLOCK_N, int SLAB_C, int EPI>
 cudaError_t launch_cfg(const ConvTcParams& p, int sm_count, cudaStream_t s) {
   using Cfg = TcCfg<BLOCK_N, SLAB_C>;
-  constexpr int SMEM = HALO ? Cfg::HALO_SMEM_BYTES : Cfg::SMEM_BYTES;
-  auto kern = conv_tc_kernel<BLOCK_N, SLAB_C, EPI, HALO>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  auto kern = conv_tc_kernel<BLOCK_N, SLAB_C, EPI>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int total_tiles = p.K * p.tiles_x * p.tiles_y * p.n_tiles_n;
   const int grid = total_tiles < sm_count ? total_tiles : sm_count;
-  kern<<<grid, TC_THREADS, SMEM, s>>>(p);
+  kern<<<grid, TC_THREADS, Cfg::SMEM_BYTES, s>>>(p);
   return cudaGetLastError();
 }
 
 template <int EPI>
 cudaError_t launch_shape(const ConvTcParams& p, int sm_count, cudaStream_t s) {
-  if (p.halo) {
-    if (p.slab_c != 64 || p.stride != 1) return cudaErrorInvalidValue;
-    if (p.block_n == 256) return launch_cfg<256, 64, EPI, true>(p, sm_count, s);
-    if (p.block_n == 128) return launch_cfg<128, 64, EPI, true>(p, sm_count, s);
-    if (p.block_n == 64) return launch_cfg<64, 64, EPI, true>(p, sm_count, s);
-    return cudaErrorInvalidValue;
-  }
   if (p.slab_c == 64) {
-    if (p.block_n == 256) return launch_cfg<256, 64, EPI, false>(p, sm_count, s);
-    if (p.block_n == 128) return launch_cfg<128, 64, EPI, false>(p, sm_count, s);
-    if (p.block_n == 64) return launch_cfg<64, 64, EPI, false>(p, sm_count, s);
+    if (p.block_n == 256) return launch_cfg<256, 64, EPI>(p, sm_count, s);
+    if (p.block_n == 128) return launch_cfg<128, 64, EPI>(p, sm_count, s);
+    if (p.block_n == 64) return launch_cfg<64, 64, EPI>(p, sm_count, s);
   } else if (p.slab_c == 32) {
-    if (p.block_n == 128) return launch_cfg<128, 32, EPI, false>(p, sm_count, s);
-    if (p.block_n == 64) return launch_cfg<64, 32, EPI, false>(p, sm_count, s);
+    if (p.block_n == 128) return launch_cfg<128, 32, EPI>(p, sm_count, s);
+    if (p.block_n == 64) return launch_cfg<64, 32, EPI>(p, sm_count, s);
   }
   return cudaErrorInvalidValue;
 }

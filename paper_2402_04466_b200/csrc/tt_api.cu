@@ -42,7 +42,6 @@ struct TcLayer {
   TensorMap128 maps_a[8];
   TensorMap128 map_b[3];       // block_n = 64, 128, 256
   bool has_b[3] = {false, false, false};
-  bool halo = false;           // stride-1 layers with 64-channel slabs: one haloed activation load per slab
 };
 
 std::mutex g_err_mu;
@@ -293,23 +292,6 @@ tt_status make_act_maps(tt_ctx* ctx, TensorMap128* maps4, __nv_bfloat16* base, i
   return TT_OK;
 }
 
-// Halo-mode activation map of one NHWC bf16 source [n_img][H][W][C] (stride 1, C a multiple of 64):
-// five dimensions (8 channels, x, y, channel group, image) with an 8 x 10 x 18 x 8 x 1 box, so one
-// load delivers eight [18][10][16-byte] planes, the no-swizzle core-matrix layout of the MMA.
-tt_status make_halo_map(tt_ctx* ctx, TensorMap128* out, __nv_bfloat16* base, int n_img, int H, int W, int C) {
-  EncodeTiledFn fn = get_encode_fn();
-  if (!fn) return fail(ctx, TT_ERR_CUDA, "cuTensorMapEncodeTiled entry point unavailable");
-  const cuuint64_t dims[5] = {8, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)(C / 8), (cuuint64_t)n_img};
-  const cuuint64_t str[4] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, 16, (cuuint64_t)H * W * C * 2};
-  const cuuint32_t box[5] = {8, 10, 18, 8, 1};
-  const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-  CUresult r = fn(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, str, box, ones,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return fail(ctx, TT_ERR_CUDA, "cuTensorMapEncodeTiled (halo map) failed with code %d", (int)r);
-  return TT_OK;
-}
-
 // OIHW fp32 -> bf16 [CoutPacked][9*Cin] with column k = tap*Cin + c.  lstm_hidden > 0: packed
 // row 4*j + gate holds original output channel gate*hidden + j.
 tt_status pack_tc(tt_ctx* ctx, TcLayer* L, const float* w, const float* b, int cin0, int cin1, int cout, int stride,
@@ -550,18 +532,10 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
     }
     TcLayer& L = ctx->tc_lstm;
     if ((st = pack_tc(ctx, &L, w->lstm_w, w->lstm_b, ctx->Cx, ctx->Ch, 4 * ctx->Ch, 1, ctx->Ch)) != TT_OK) return st;
-    L.halo = L.slab_c == 64;
-    if (L.halo) {
-      if ((st = make_halo_map(ctx, &L.maps_a[0], reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[c.n_enc - 1]), S, ctx->Hm, ctx->Wm,
-                              ctx->Cx)) != TT_OK)
-        return st;
-      if ((st = make_halo_map(ctx, &L.maps_a[4], ctx->h_bf16, 2 * S, ctx->Hm, ctx->Wm, ctx->Ch)) != TT_OK) return st;
-    } else {
-      if ((st = make_act_maps(ctx, &L.maps_a[0], reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[c.n_enc - 1]), S, ctx->Hm,
-                              ctx->Wm, ctx->Cx, 1, L.slab_c)) != TT_OK)
-        return st;
-      if ((st = make_act_maps(ctx, &L.maps_a[4], ctx->h_bf16, 2 * S, ctx->Hm, ctx->Wm, ctx->Ch, 1, L.slab_c)) != TT_OK) return st;
-    }
+    if ((st = make_act_maps(ctx, &L.maps_a[0], reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[c.n_enc - 1]), S, ctx->Hm,
+                            ctx->Wm, ctx->Cx, 1, L.slab_c)) != TT_OK)
+      return st;
+    if ((st = make_act_maps(ctx, &L.maps_a[4], ctx->h_bf16, 2 * S, ctx->Hm, ctx->Wm, ctx->Ch, 1, L.slab_c)) != TT_OK) return st;
   }
   for (int i = 0; i < TT_MAX_STREAMS; ++i) {
     ctx->states[i].ctx = ctx;
@@ -676,9 +650,8 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
     }
     auto fill_common = [&](ConvTcParams& q, const TcLayer& L, int Ho, int Wo) -> tt_status {
       std::memcpy(q.maps_a, L.maps_a, sizeof(q.maps_a));
-      q.slab_c = L.slab_c; q.stride = L.stride; q.K = K; q.Ho = Ho; q.Wo = Wo; q.halo = L.halo ? 1 : 0;
-      q.tiles_x = L.halo ? (Wo + 7) / 8 : (Wo + 15) / 16;
-      q.tiles_y = L.halo ? (Ho + 15) / 16 : (Ho + 7) / 8;
+      q.slab_c = L.slab_c; q.stride = L.stride; q.K = K; q.Ho = Ho; q.Wo = Wo;
+      q.tiles_x = (Wo + 15) / 16; q.tiles_y = (Ho + 7) / 8;
       const int bi = pick_block_n(L, K * q.tiles_x * q.tiles_y, ctx->sm_count);
       if (bi < 0) return fail(ctx, TT_ERR_UNSUPPORTED, "no tensor-core tile shape fits this layer");
       const int bns[3] = {64, 128, 256};

@@ -102,7 +102,6 @@ struct ConvTcParams {
   int32_t slabs[2];         // channel slabs (of slab_c channels) per source
   int32_t slab_c;           // 64 or 32
   int32_t stride;           // 1 or 2
-  int32_t halo;             // 1: stride-1 halo mode (8 x 16 patch, one haloed activation load per channel slab)
   int32_t K;                // images in the batch
   IdxMap img0, img1;        // image index of batch n inside source 0 / 1
   int32_t Ho, Wo;           // output extent
