@@ -72,6 +72,8 @@ __global__ void __launch_bounds__(TW* TH) conv3x3_simt_kernel(const __grid_const
       if (ci < cin && yi >= 0 && yi < p.H && xi >= 0 && xi < p.W) {
         const float* src = ci < p.C0 ? base0 + (size_t)ci * in_plane : base1 + (size_t)(ci - p.C0) * in_plane;
         v = __ldg(src + (size_t)yi * p.W + xi);
+        // on the bf16 path every contraction takes bf16 operands, like the tensor-core layers
+        if (EPI == EPI_RELU_BF16_NHWC) v = __bfloat162float(__float2bfloat16_rn(v));
       }
       s_in[(c * IN_H + r) * IN_WP + col] = v;
     }

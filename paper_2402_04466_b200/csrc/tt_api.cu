@@ -107,9 +107,7 @@ struct tt_ctx {
   float *head_w = nullptr, *head_b = nullptr, *conf_w = nullptr, *conf_b = nullptr;
   float zthr = 0.f;
 
-  ConvFirstParams first{};      // bf16 path, first encoder layer when its width is supported
-  bool use_first = false;
-  ConvFirstTcParams first_tc{}; // ... on the tensor cores when its width allows
+  ConvFirstTcParams first_tc{}; // bf16 path, first encoder layer on the tensor cores when its width (32 or 64) allows
   bool use_first_tc = false;
   SimtLayer simt_enc[TT_MAX_ENC];
   SimtLayer simt_lstm;
@@ -506,19 +504,6 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
         if ((st = encode_map(ctx, &f.map_out, ctx->enc_out[0], 4, dims, str, box, co * 2)) != TT_OK) return st;
       }
       ctx->use_first_tc = true;
-    } else if (conv_first_supported(ctx->lay_c[1])) {
-      ConvFirstParams& f = ctx->first;
-      const int co = ctx->lay_c[1];
-      f.in = ctx->pre; f.out = reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[0]);
-      f.H = c.net_h; f.W = c.net_w; f.Ho = ctx->lay_h[1]; f.Wo = ctx->lay_w[1]; f.stride = c.enc_stride[0]; f.cout = co;
-      for (int o = 0; o < co; ++o) {
-        f.b[o] = w->enc_b[0][o];
-        for (int t = 0; t < 27; ++t) {
-          uint32_t u = (uint32_t)f32_to_bf16_rne(w->enc_w[0][(size_t)o * 27 + t]) << 16;
-          std::memcpy(&f.w[t * co + o], &u, 4);
-        }
-      }
-      ctx->use_first = true;
     } else if ((st = pack_simt(ctx, &ctx->simt_enc[0], w->enc_w[0], w->enc_b[0], 3, ctx->lay_c[1], c.enc_stride[0],
                                ctx->lay_c[1] > 16 ? 32 : 16, 0, true)) != TT_OK) {
       return st;
@@ -632,10 +617,6 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
     if (ctx->use_first_tc) {
       ctx->first_tc.K = K;
       TT_CUDA(ctx, launch_conv_first_tc(ctx->first_tc, ctx->sm_count, s));
-      if ((ms_ = mark_stage(ctx, TT_STAGE_ENC0, 1)) != TT_OK) return ms_;
-    } else if (ctx->use_first) {
-      ctx->first.K = K;
-      TT_CUDA(ctx, launch_conv_first(ctx->first, s));
       if ((ms_ = mark_stage(ctx, TT_STAGE_ENC0, 1)) != TT_OK) return ms_;
     } else {
       const SimtLayer& L = ctx->simt_enc[0];

@@ -62,19 +62,7 @@ struct alignas(64) TensorMap128 {
 };
 
 // --------------------------------------- S2 first encoder layer of the bf16 path (Cin = 3)
-// Passed by value: the weights sit in the kernel parameter block (constant bank).
-constexpr int CONV_FIRST_MAX_COUT = 64;
-struct ConvFirstParams {
-  const float* in;       // [K][3][H][W] fp32
-  __nv_bfloat16* out;    // [K][Ho][Wo][cout] bf16
-  int32_t H, W, Ho, Wo, stride, K, cout;
-  float w[27 * CONV_FIRST_MAX_COUT];  // [(c*3+ky)*3+kx][cout]
-  float b[CONV_FIRST_MAX_COUT];
-};
-bool conv_first_supported(int cout);
-cudaError_t launch_conv_first(const ConvFirstParams& p, cudaStream_t s);
-
-// Same layer on the tensor cores (cout 32 or 64): operand tiles are built by gather threads.
+// On the tensor cores (cout 32 or 64): operand tiles are built by producer threads.
 struct ConvFirstTcParams {
   TensorMap128 map_out;       // output [K][Ho][Wo][cout] bf16, box [cout][16][8][1], 128B / 64B swizzle
   const float* in;            // [K][3][H][W] fp32

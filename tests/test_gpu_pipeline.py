@@ -166,6 +166,14 @@ def test_bf16_odd_extents_on_strided_layers(cuda_device):
     _run_bf16(cuda_device, wl, 2, 3)
 
 
+def test_bf16_first_layer_width_outside_the_tensor_core_kernel(cuda_device):
+    """A first layer of 96 channels is not covered by the tensor-core first-layer kernel: the fp32 SIMT kernel writes
+    the bf16 channels-last map instead, and the next layer runs on 32-channel slabs."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="bf16-96", src_w=120, src_h=90, net_w=96, net_h=72,
+                                              enc_cout=(96, 64), enc_stride=(2, 2), hidden=32)
+    _run_bf16(cuda_device, wl, 2, 2)
+
+
 def test_bf16_wide_channels_small_map(cuda_device):
     """The scale-sweep channel widths (64/128/256, hidden 256: N = 1024, K = 4608) on a small map."""
     wl = tt_synth.workload("cfg4-gain").with_(name="bf16-wide", src_w=160, src_h=120, net_w=136, net_h=104)
