@@ -33,7 +33,7 @@ __device__ __forceinline__ uint32_t blend_px(int r, int g, int b, uint32_t bits,
 template <bool PACKED, bool FLAT>
 __global__ void __launch_bounds__(256) overlay_kernel(const __grid_constant__ OverlayParams p) {
   const int n = blockIdx.y;
-  const uint8_t* __restrict__ src = p.src.p[n];
+  const uint8_t* __restrict__ src = p.src_tab ? p.src_tab[n] : p.src.p[n];
   const long long npx = (long long)p.src_w * p.src_h;
   uint8_t* dst = p.dst + (size_t)n * npx * 4;
   const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;  // group of 4 pixels

@@ -74,7 +74,7 @@ preprocess_staged_kernel(const __grid_constant__ PreprocessParams p, int row_cap
   __shared__ float s_fy[PRE_ROWS];
   __shared__ int s_xlo, s_xhi;                       // source column range of the tile
   const int n = blockIdx.z;
-  const uint8_t* __restrict__ src = p.src.p[n];
+  const uint8_t* __restrict__ src = p.src_tab ? p.src_tab[n] : p.src.p[n];
   const uint32_t src_lo = (uint32_t)(uintptr_t)src;  // only the low bits matter for 16-byte alignment
   const int xo_blk = blockIdx.x * PRE_OUT_W;
   const int yo_blk = blockIdx.y * PRE_ROWS;
@@ -171,7 +171,7 @@ preprocess_staged_kernel(const __grid_constant__ PreprocessParams p, int row_cap
 // taps are read straight from global memory (L1-cached byte loads).
 __global__ void __launch_bounds__(PRE_THREADS) preprocess_direct_kernel(const __grid_constant__ PreprocessParams p, float scale, float shift) {
   const int n = blockIdx.z;
-  const uint8_t* __restrict__ src = p.src.p[n];
+  const uint8_t* __restrict__ src = p.src_tab ? p.src_tab[n] : p.src.p[n];
   const int yo = blockIdx.y * PRE_TY + threadIdx.y;
   const int xo0 = blockIdx.x * PRE_OUT_W + threadIdx.x * 4;
   if (yo >= p.net_h || xo0 >= p.net_w) return;

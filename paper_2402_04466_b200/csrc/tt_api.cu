@@ -135,6 +135,21 @@ struct tt_ctx {
   int q_head = 0, q_count = 0;      // oldest in-flight slot, number in flight
   int bound = 0;                    // slot whose resources the view members hold
   int last_done = -1;               // slot of the last completed submit (debug taps)
+  // CUDA graphs of the tick's launch sequence, one per (stream count, slot, state placement).  Frame
+  // pointers change every tick, so the kernels read them from a small device table per slot that
+  // is refreshed by a 64-byte copy in front of the graph launch.
+  struct TickGraph {
+    int K = 0, slot = 0, flat = 0;
+    int sig[TT_MAX_STREAMS] = {};   // state slot * 2 + half of every batch position
+    int seen = 0;                   // direct executions of this key so far (capture happens on the second)
+    uint64_t launches = 0;          // kernels inside the graph
+    cudaGraphExec_t exec = nullptr;
+  };
+  std::vector<TickGraph> graphs;
+  bool graphs_off = false;
+  const uint8_t** frame_tab_dev[2] = {nullptr, nullptr};   // device, [TT_MAX_STREAMS] pointers per slot
+  const uint8_t** frame_tab_host[2] = {nullptr, nullptr};  // pinned staging of the same
+  const uint8_t* const* cur_tab = nullptr;                  // table the tick being enqueued reads
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_copy = nullptr;
   bool tick_profiled = false;
@@ -451,12 +466,19 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
     TT_CUDA(ctx, cudaHostAlloc(reinterpret_cast<void**>(&sl.results_host), sizeof(tt_result) * S, cudaHostAllocDefault));
     TT_CUDA(ctx, cudaHostAlloc(reinterpret_cast<void**>(&sl.status_host), sizeof(int32_t), cudaHostAllocDefault));
     *sl.status_host = 0;
+    {
+      uint64_t* tab = nullptr;
+      if ((st = dev_alloc(ctx, &tab, (size_t)TT_MAX_STREAMS)) != TT_OK) return st;
+      ctx->frame_tab_dev[i] = reinterpret_cast<const uint8_t**>(tab);
+      TT_CUDA(ctx, cudaHostAlloc(reinterpret_cast<void**>(&ctx->frame_tab_host[i]), sizeof(void*) * TT_MAX_STREAMS, cudaHostAllocDefault));
+    }
     TT_CUDA(ctx, cudaEventCreate(&sl.ev_start));
     TT_CUDA(ctx, cudaEventCreate(&sl.ev_stop));
     TT_CUDA(ctx, cudaEventCreateWithFlags(&sl.ev_copy, cudaEventDisableTiming));
     for (int k = 0; k <= TT_STAGE_COUNT; ++k) TT_CUDA(ctx, cudaEventCreate(&sl.stage_ev[k]));
   }
   bind_slot(ctx, 0);
+  ctx->graphs_off = c.reserved_[0] != 0;
 
   // ---- weights
   const bool r = ctx->bf16;  // round weights to bf16 on the bf16 path
@@ -546,6 +568,10 @@ void release(tt_ctx* ctx) {
     for (int k = 0; k <= TT_STAGE_COUNT; ++k)
       if (sl.stage_ev[k]) cudaEventDestroy(sl.stage_ev[k]);
   }
+  for (auto& g : ctx->graphs)
+    if (g.exec) cudaGraphExecDestroy(g.exec);
+  for (int i = 0; i < 2; ++i)
+    if (ctx->frame_tab_host[i]) cudaFreeHost(ctx->frame_tab_host[i]);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   if (ctx->own_stream && ctx->stream) cudaStreamDestroy(ctx->stream);
   delete ctx;
@@ -581,7 +607,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
   }
 
   PreprocessParams pp;
-  pp.src = frames; pp.K = K; pp.src_w = c.src_w; pp.src_h = c.src_h; pp.src_pitch = c.src_pitch;
+  pp.src = frames; pp.src_tab = ctx->cur_tab; pp.K = K; pp.src_w = c.src_w; pp.src_h = c.src_h; pp.src_pitch = c.src_pitch;
   pp.net_w = c.net_w; pp.net_h = c.net_h;
   pp.inv_div = 1.0f / c.norm_div; pp.mean = c.norm_mean; pp.inv_std = 1.0f / c.norm_std;
   pp.dst = ctx->pre;
@@ -674,7 +700,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
 
   if (c.overlay) {
     OverlayParams ov{};
-    ov.src = frames; ov.K = K; ov.src_w = c.src_w; ov.src_h = c.src_h; ov.src_pitch = c.src_pitch;
+    ov.src = frames; ov.src_tab = ctx->cur_tab; ov.K = K; ov.src_w = c.src_w; ov.src_h = c.src_h; ov.src_pitch = c.src_pitch;
     ov.T = ctx->T; ov.Hm = ctx->Hm; ov.Wm = ctx->Wm; ov.masks = ctx->masks; ov.bits = ctx->bits;
     std::memcpy(ov.palette, c.palette, sizeof(ov.palette));
     ov.dst = ctx->overlay;
@@ -855,10 +881,80 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
     st = mark_stage(ctx, TT_STAGE_H2D, 0);
     if (st != TT_OK) return st;
   }
-  st = enqueue_tick(ctx, K, fp, states);
-  if (st != TT_OK) return st;
-  TT_CUDA(ctx, cudaMemcpyAsync(ctx->results_host, ctx->results_dev, sizeof(tt_result) * K, cudaMemcpyDeviceToHost, s));
-  TT_CUDA(ctx, cudaMemcpyAsync(ctx->status_host, ctx->status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  // frame pointers of this tick -> the slot's device table (the kernels read them from there)
+  for (int n = 0; n < TT_MAX_STREAMS; ++n) ctx->frame_tab_host[slot][n] = n < K ? fp.p[n] : nullptr;
+  TT_CUDA(ctx, cudaMemcpyAsync(ctx->frame_tab_dev[slot], ctx->frame_tab_host[slot], sizeof(void*) * TT_MAX_STREAMS,
+                               cudaMemcpyHostToDevice, s));
+  ctx->cur_tab = ctx->frame_tab_dev[slot];
+
+  // The launch sequence of a tick is replayed from a CUDA graph once the same (K, slot, state
+  // placement) has been seen before; the first occurrence runs as plain launches.  With stage
+  // events requested the tick always runs as plain launches.
+  tt_ctx::TickGraph* tg = nullptr;
+  if (!ctx->graphs_off && !ctx->profiling) {
+    int flat = 1;
+    // the overlay launch picks its word-wise variant from the frames' 4-byte alignment: part of the key
+    for (int n = 0; n < K; ++n) flat &= (((uintptr_t)fp.p[n] & 3) == 0) ? 1 : 0;
+    for (auto& g : ctx->graphs) {
+      bool same = g.K == K && g.slot == slot && g.flat == flat;
+      for (int n = 0; n < K && same; ++n) same = g.sig[n] == states[n]->slot * 2 + states[n]->half;
+      if (same) { tg = &g; break; }
+    }
+    if (!tg) {
+      if (ctx->graphs.size() >= 64) {            // bounded cache: drop everything and start over
+        for (auto& g : ctx->graphs)
+          if (g.exec) cudaGraphExecDestroy(g.exec);
+        ctx->graphs.clear();
+      }
+      tt_ctx::TickGraph g;
+      g.K = K; g.slot = slot; g.flat = flat;
+      for (int n = 0; n < K; ++n) g.sig[n] = states[n]->slot * 2 + states[n]->half;
+      ctx->graphs.push_back(g);
+      tg = &ctx->graphs.back();
+    }
+  }
+  if (tg && tg->exec) {
+    TT_CUDA(ctx, cudaGraphLaunch(tg->exec, s));
+    ctx->n_launches += tg->launches;
+    ctx->n_ticks += 1;
+  } else if (tg && tg->seen >= 1) {
+    // second occurrence: capture the sequence (kernels plus the two result copies), then launch it
+    const uint64_t launches_before = ctx->n_launches;
+    cudaGraph_t graph = nullptr;
+    cudaError_t ce = cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal);
+    if (ce == cudaSuccess) {
+      st = enqueue_tick(ctx, K, fp, states);
+      if (st == TT_OK) {
+        ce = cudaMemcpyAsync(ctx->results_host, ctx->results_dev, sizeof(tt_result) * K, cudaMemcpyDeviceToHost, s);
+        if (ce == cudaSuccess) ce = cudaMemcpyAsync(ctx->status_host, ctx->status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, s);
+      }
+      cudaError_t ee = cudaStreamEndCapture(s, &graph);
+      if (ce == cudaSuccess) ce = ee;
+    }
+    if (st == TT_OK && ce == cudaSuccess && graph) ce = cudaGraphInstantiate(&tg->exec, graph, 0);
+    if (graph) cudaGraphDestroy(graph);
+    if (st != TT_OK || ce != cudaSuccess || !tg->exec) {
+      // capture is an optimisation only: clear the error, switch it off and run this tick directly
+      cudaGetLastError();
+      tg->exec = nullptr;
+      ctx->graphs_off = true;
+      ctx->n_launches = launches_before;
+      ctx->n_ticks -= (st == TT_OK) ? 1 : 0;
+      st = enqueue_tick(ctx, K, fp, states);
+      if (st != TT_OK) return st;
+      TT_CUDA(ctx, cudaMemcpyAsync(ctx->results_host, ctx->results_dev, sizeof(tt_result) * K, cudaMemcpyDeviceToHost, s));
+      TT_CUDA(ctx, cudaMemcpyAsync(ctx->status_host, ctx->status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    } else {
+      tg->launches = ctx->n_launches - launches_before;
+      TT_CUDA(ctx, cudaGraphLaunch(tg->exec, s));
+    }
+  } else {
+    st = enqueue_tick(ctx, K, fp, states);
+    if (st != TT_OK) return st;
+    TT_CUDA(ctx, cudaMemcpyAsync(ctx->results_host, ctx->results_dev, sizeof(tt_result) * K, cudaMemcpyDeviceToHost, s));
+    TT_CUDA(ctx, cudaMemcpyAsync(ctx->status_host, ctx->status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    if (tg) tg->seen += 1;
+  }
   TT_CUDA(ctx, cudaEventRecord(ctx->ev_stop, s));
   for (int n = 0; n < TT_MAX_STREAMS; ++n) ctx->states[n].last_pos = -1;
   for (int n = 0; n < K; ++n) {

@@ -21,7 +21,8 @@ struct FramePtrs {
 
 // ------------------------------------------------------------------------- S1 preprocess
 struct PreprocessParams {
-  FramePtrs src;
+  FramePtrs src;                   // frame pointers by value (also used for host-side decisions)
+  const uint8_t* const* src_tab;   // if non-null the kernel reads the pointers from this device table instead
   int32_t K, src_w, src_h, src_pitch, net_w, net_h;
   float inv_div, mean, inv_std;
   float* dst;  // [K][3][net_h][net_w]
@@ -140,6 +141,7 @@ cudaError_t post_static_scratch(void** ptr);  // device address of the library's
 // -------------------------------------------------------------------------- S6 overlay
 struct OverlayParams {
   FramePtrs src;
+  const uint8_t* const* src_tab;   // as in PreprocessParams
   int32_t K, src_w, src_h, src_pitch, T, Hm, Wm;
   const uint8_t* masks;  // [K][T][plane] (used when bits == null)
   const uint8_t* bits;   // [K][plane] packed

@@ -13,9 +13,10 @@ from parity_util import assert_close, check_masks, check_reductions_from_own_mas
 pytestmark = pytest.mark.gpu
 
 
-def _make(wl, K=1, overlay=None, precision=None, timeout_ns=0):
+def _make(wl, K=1, overlay=None, precision=None, timeout_ns=0, plain_launches=False):
     weights = tt_synth.make_weights(wl)
-    cfg = binding.make_config(wl, max_streams=K, overlay=overlay, precision=precision, sync_timeout_ns=timeout_ns)
+    cfg = binding.make_config(wl, max_streams=K, overlay=overlay, precision=precision, sync_timeout_ns=timeout_ns,
+                              plain_launches=plain_launches)
     ctx = binding.Context(cfg, weights)
     states = [ctx.state_create() for _ in range(K)]
     return ctx, states, weights
@@ -273,6 +274,61 @@ def test_runs_are_bitwise_reproducible(cuda_device):
     for k in range(K):
         assert np.array_equal(outs[0][0][k][0], outs[1][0][k][0]) and np.array_equal(outs[0][0][k][1], outs[1][0][k][1])
         assert np.array_equal(outs[0][1][k], outs[1][1][k]) and np.array_equal(outs[0][2][k], outs[1][2][k])
+
+
+def test_graph_replay_matches_plain_launches(cuda_device):
+    """A tick replayed from a captured graph must give bit for bit what kernel-by-kernel launches give, while
+    the batch size, the set of active streams and the frames' addresses (4-byte aligned or not, which selects
+    the overlay variant) change from tick to tick and both submit slots are in use."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="graph", src_w=214, src_h=120, net_w=160, net_h=120, overlay=True)
+    K, n = 3, 14
+    host = _frames(wl, K, n)
+    nbytes = host[0][0].size
+    # every frame twice on the device: once 4-byte aligned, once at an odd byte offset
+    bufs = [[torch.empty(nbytes + 16, dtype=torch.uint8, device=cuda_device) for _ in range(2 * n)] for _ in range(K)]
+    shape = host[0][0].shape
+
+    def frame(k, t, odd):
+        b = bufs[k][2 * t + int(odd)]
+        v = b[1:1 + nbytes] if odd else b[:nbytes]
+        v.copy_(torch.from_numpy(host[k][t]).reshape(-1))
+        return v.view(shape)
+
+    # which streams take part in tick t, and whether stream 0's frame sits at an odd address
+    plan = [((0, 1, 2), False)] * 4 + [((0, 2), False)] * 3 + [((0, 1, 2), True)] * 3 + [((1,), False)] * 2 + [((0, 1, 2), False)] * 2
+    assert len(plan) == n
+    runs = []
+    for plain in (True, False):
+        ctx, states, _ = _make(wl, K, overlay=True, plain_launches=plain)
+        out = []
+        pending = 0
+        for t, (who, odd) in enumerate(plan):
+            ctx.submit_frames([frame(k, t, odd and k == 0) for k in who], [states[k] for k in who], frame_index=t)
+            pending += 1
+            if pending == 2:
+                r = ctx.sync()
+                out.append([(x["frame_index"], ctx.fetch_probs(x), ctx.fetch_overlay(x), x["conf"].copy(), x["cx"].copy(),
+                             x["count"].copy()) for x in r])
+                pending -= 1
+        while pending:
+            r = ctx.sync()
+            out.append([(x["frame_index"], ctx.fetch_probs(x), ctx.fetch_overlay(x), x["conf"].copy(), x["cx"].copy(),
+                         x["count"].copy()) for x in r])
+            pending -= 1
+        launches, ticks = ctx.get_counters()
+        runs.append((out, [ctx.state_export(s) for s in states], ticks, launches))
+        ctx.destroy()
+    (a, ha, ta, la), (b, hb, tb, lb) = runs
+    assert ta == tb == n and la == lb, "replayed ticks must count the launches they contain"
+    assert len(a) == len(b) == n
+    for ra, rb in zip(a, b):
+        assert len(ra) == len(rb)
+        for xa, xb in zip(ra, rb):
+            assert xa[0] == xb[0]
+            for va, vb in zip(xa[1:], xb[1:]):
+                assert np.array_equal(va, vb)
+    for (h1, c1), (h2, c2) in zip(ha, hb):
+        assert np.array_equal(h1, h2) and np.array_equal(c1, c2)
 
 
 def test_two_submits_in_flight_match_serial_execution(cuda_device):
