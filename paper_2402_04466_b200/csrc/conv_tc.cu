@@ -13,9 +13,14 @@
 // columns), each an ordinary tiled tensor map with doubled strides, so every tap is again
 // a dense box.
 //
-// Warp roles (320 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM allocation and
-// MMA issue (one lane), warps 2..9 = epilogue (TMEM lane quarter = warp index mod 4, two warps
-// per quarter, each taking half of the tile's columns).
+// Warp roles (384 threads): warp 0 and warps 10, 11 = TMA producers (one lane each; producer j
+// issues the loads of pipeline iterations j, j + n_prod, ... so that the cost of issuing a copy is
+// spread over several instruction streams), warp 1 = TMEM allocation and MMA issue (one lane),
+// warps 2..9 = epilogue (TMEM lane quarter = warp index mod 4, two warps per quarter, each taking
+// half of the tile's columns).  The single threads that issue copies and MMAs are latency-bound
+// instruction streams, so the roles are laid out so that each of them sits on a different warp
+// scheduler (warp index mod 4).  What a pipeline iteration loads (tensor map, channel offset, tap
+// shift) is the same for every tile, so it is tabulated in shared memory once per block.
 // Every mbarrier wait is bounded: when a wait runs out the kernel records a status code,
 // raises a block-wide abort flag, lets copies in flight land, frees its TMEM and returns.
 #include "tt_internal.h"
@@ -30,7 +35,11 @@ constexpr int BLOCK_M = 128;
 constexpr int PATCH_W = 16, PATCH_H = 8;
 constexpr int UMMA_K = 16;
 constexpr int EPI_WARPS = 8;                       // two per TMEM lane quarter, each takes half of the columns
-constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;
+constexpr int N_PROD = 3;                          // producer warps: 0, 10, 11
+constexpr int MMA_WARP = 1;
+constexpr int EPI_WARP0 = 2;
+constexpr int TC_THREADS = 32 * (2 + EPI_WARPS + (N_PROD - 1));
+constexpr int MAX_K_ITERS = 9 * 16;                // 9 taps x up to 16 channel slabs
 
 template <int BLOCK_N, int SLAB_C>
 struct TcCfg {
@@ -41,7 +50,9 @@ struct TcCfg {
   static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
   static constexpr int TMEM_COLS = 2 * BLOCK_N < 32 ? 32 : 2 * BLOCK_N;
   static constexpr int BAR_BYTES = 256;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024 /*alignment slack*/;
+  static constexpr int TAB_BYTES = MAX_K_ITERS * 16 + 4 * TT_MAX_STREAMS * 4;   // iteration table + image index maps
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + TAB_BYTES + 1024 /*alignment slack*/;
+  static_assert(STAGES >= N_PROD, "every producer needs a stage of its own");
   static_assert((TMEM_COLS & (TMEM_COLS - 1)) == 0 && TMEM_COLS <= 512, "TMEM columns must be a power of two <= 512");
   static_assert(A_BYTES % 1024 == 0 && B_BYTES % 1024 == 0, "operand tiles must keep 1024-byte alignment");
 };
@@ -74,8 +85,43 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
   uint64_t* tempty_bar = tfull_bar + 2;                        // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int4* s_tab = reinterpret_cast<int4*>(bar_mem + Cfg::BAR_BYTES);            // [k_iters] {map slot, channel offset, dx, dy}
+  int* s_img = reinterpret_cast<int*>(s_tab + MAX_K_ITERS);                   // [4][TT_MAX_STREAMS]: img0, img1, c_idx, h_out_idx
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_per_img = p.tiles_x * p.tiles_y;
+  const int total_tiles = p.K * tiles_per_img * p.n_tiles_n;
+  const int slabs_per_tap = p.slabs[0] + (p.n_src > 1 ? p.slabs[1] : 0);
+  const int k_iters = 9 * slabs_per_tap;
+
+  // What iteration `it` of a tile's main loop loads: tap it / slabs_per_tap, then source x
+  // before source h, then the channel slab.
+  for (int it = threadIdx.x; it < k_iters; it += TC_THREADS) {
+    const int tap = it / slabs_per_tap, r = it % slabs_per_tap;
+    const int src = r < p.slabs[0] ? 0 : 1;
+    const int sl = src ? r - p.slabs[0] : r;
+    const int ky = tap / 3, kx = tap % 3;
+    int dx, dy, par;
+    if (p.stride == 1) {
+      dx = kx - 1;
+      dy = ky - 1;
+      par = 0;
+    } else {
+      // input column 2*xo + kx - 1: kx = 1 is the even view at xo, kx = 0 / 2 the odd view at xo-1 / xo
+      const int xpar = (kx == 1) ? 0 : 1, ypar = (ky == 1) ? 0 : 1;
+      dx = kx == 0 ? -1 : 0;
+      dy = ky == 0 ? -1 : 0;
+      par = ypar * 2 + xpar;
+    }
+    s_tab[it] = make_int4(src * 4 + par, sl * SLAB_C, dx, dy);
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&p.maps_a[src * 4 + par]) : "memory");
+  }
+  if (threadIdx.x < TT_MAX_STREAMS) {
+    s_img[threadIdx.x] = p.img0.v[threadIdx.x];
+    s_img[TT_MAX_STREAMS + threadIdx.x] = p.img1.v[threadIdx.x];
+    s_img[2 * TT_MAX_STREAMS + threadIdx.x] = p.c_idx.v[threadIdx.x];
+    s_img[3 * TT_MAX_STREAMS + threadIdx.x] = p.h_out_idx.v[threadIdx.x];
+  }
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -88,8 +134,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&p.map_b) : "memory");
   }
-  if (warp == 1) {
+  if (warp == MMA_WARP) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                  "r"((uint32_t)Cfg::TMEM_COLS)
                  : "memory");
@@ -100,53 +147,37 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int tiles_per_img = p.tiles_x * p.tiles_y;
-  const int total_tiles = p.K * tiles_per_img * p.n_tiles_n;
-  const int slabs_per_tap = p.slabs[0] + (p.n_src > 1 ? p.slabs[1] : 0);
-  const int k_iters = 9 * slabs_per_tap;
-
-  if (warp == 0 && lane == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    uint32_t stage = 0, phase = 0;
+  const int n_prod = p.n_prod;
+  const int prod = warp == 0 ? 0 : warp - (EPI_WARP0 + EPI_WARPS) + 1;   // producer index of warps 0, 10, 11
+  if ((warp == 0 || warp >= EPI_WARP0 + EPI_WARPS) && prod < n_prod && lane == 0) {
+    // ----------------------------------------------------------------- TMA producers
+    // Producer `prod` owns iterations prod, prod + n_prod, ... of the block's sequence of
+    // pipeline iterations (all tiles back to back); iteration g uses stage g % STAGES.
+    uint32_t stage = (uint32_t)prod % STAGES, phase = 0;
+    int it = prod;
     bool ok = true;
+    const uint8_t* maps = reinterpret_cast<const uint8_t*>(p.maps_a);
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int nt = tile % p.n_tiles_n;
       const int m = tile / p.n_tiles_n;
       const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
       const int x0 = tx * PATCH_W, y0 = ty * PATCH_H;
-      int kcol = 0;
-      for (int tap = 0; tap < 9 && ok; ++tap) {
-        const int ky = tap / 3, kx = tap % 3;
-        int cx, cy, par;
-        if (p.stride == 1) {
-          cx = x0 + kx - 1;
-          cy = y0 + ky - 1;
-          par = 0;
-        } else {
-          // input column 2*xo + kx - 1: kx = 1 is the even view at xo, kx = 0 / 2 the odd view at xo-1 / xo
-          const int xpar = (kx == 1) ? 0 : 1, ypar = (ky == 1) ? 0 : 1;
-          cx = x0 + (kx == 0 ? -1 : 0);
-          cy = y0 + (ky == 0 ? -1 : 0);
-          par = ypar * 2 + xpar;
-        }
-        for (int src = 0; src < p.n_src && ok; ++src) {
-          const void* map_a = &p.maps_a[src * 4 + par];
-          const int img_idx = src == 0 ? p.img0.v[img] : p.img1.v[img];
-          for (int sl = 0; sl < p.slabs[src]; ++sl) {
-            ok = mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag, p.status, 0x100 + (int)stage);
-            if (!ok) break;
-            const uint32_t fb = smem_u32(full_bar + stage);
-            uint8_t* st = smem + stage * Cfg::STAGE_BYTES;
-            mbar_arrive_expect_tx(fb, Cfg::STAGE_BYTES);
-            tma_load_4d(smem_u32(st), map_a, fb, sl * SLAB_C, cx, cy, img_idx);
-            tma_load_2d(smem_u32(st + Cfg::A_BYTES), &p.map_b, fb, kcol, nt * BLOCK_N);
-            kcol += SLAB_C;
-            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-          }
-        }
+      const int img_a[2] = {s_img[img], s_img[TT_MAX_STREAMS + img]};
+      for (; it < k_iters; it += n_prod) {
+        const int4 e = s_tab[it];
+        ok = mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag, p.status, 0x100 + (int)stage);
+        if (!ok) break;
+        const uint32_t fb = smem_u32(full_bar + stage);
+        uint8_t* st = smem + stage * Cfg::STAGE_BYTES;
+        mbar_arrive_expect_tx(fb, Cfg::STAGE_BYTES);
+        tma_load_4d(smem_u32(st), maps + e.x * (int)sizeof(TensorMap128), fb, e.y, x0 + e.z, y0 + e.w, img_a[e.x >> 2]);
+        tma_load_2d(smem_u32(st + Cfg::A_BYTES), &p.map_b, fb, it * SLAB_C, nt * BLOCK_N);
+        stage += (uint32_t)n_prod;
+        if (stage >= (uint32_t)STAGES) { stage -= STAGES; phase ^= 1u; }
       }
+      it -= k_iters;
     }
-  } else if (warp == 1 && lane == 0) {
+  } else if (warp == MMA_WARP && lane == 0) {
     // -------------------------------------------------------------------- MMA issuer
     uint32_t stage = 0, phase = 0, acc_phase = 0;
     int acc = 0;
@@ -176,12 +207,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
       umma_commit(smem_u32(tfull_bar + acc));      // accumulator complete
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
-  } else if (warp >= 2) {
+  } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + EPI_WARPS) {
     // ---------------------------------------------------------------------- epilogue
     constexpr int HALF_N = BLOCK_N / 2;           // columns handled by this warp
     constexpr int CHUNKS = HALF_N / 32;
     const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
-    const int half = (warp - 2) >> 2;             // which half of the tile's columns
+    const int half = (warp - EPI_WARP0) >> 2;     // which half of the tile's columns
     const int row = quarter * 32 + lane;          // row of the 128-row tile = pixel of the patch
     const int py = row / PATCH_W, px = row % PATCH_W;
     uint32_t acc_phase = 0;
@@ -201,8 +232,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
       float c_old[EPI == TC_EPI_LSTM ? CHUNKS * 8 : 1];
       size_t so = 0, ho = 0;
       if (EPI == TC_EPI_LSTM) {
-        so = ((size_t)p.c_idx.v[img] * p.Ho * p.Wo + pix) * p.hidden + (col0 >> 2);
-        ho = ((size_t)p.h_out_idx.v[img] * p.Ho * p.Wo + pix) * p.hidden + (col0 >> 2);
+        so = ((size_t)s_img[2 * TT_MAX_STREAMS + img] * p.Ho * p.Wo + pix) * p.hidden + (col0 >> 2);
+        ho = ((size_t)s_img[3 * TT_MAX_STREAMS + img] * p.Ho * p.Wo + pix) * p.hidden + (col0 >> 2);
 #pragma unroll
         for (int ck = 0; ck < CHUNKS; ++ck) {
           float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
@@ -286,7 +317,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == MMA_WARP) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS)
                  : "memory");
@@ -323,6 +354,7 @@ cudaError_t launch_shape(const ConvTcParams& p, int sm_count, cudaStream_t s) {
 cudaError_t conv_tc_prepare() { return cudaSuccess; }
 
 cudaError_t launch_conv_tc(const ConvTcParams& p, int sm_count, cudaStream_t s) {
+  if (9 * (p.slabs[0] + (p.n_src > 1 ? p.slabs[1] : 0)) > MAX_K_ITERS || p.n_prod < 1 || p.n_prod > N_PROD) return cudaErrorInvalidValue;
   if (p.epilogue == TC_EPI_RELU_BF16) return launch_shape<TC_EPI_RELU_BF16>(p, sm_count, s);
   if (p.epilogue == TC_EPI_LSTM) return launch_shape<TC_EPI_LSTM>(p, sm_count, s);
   return cudaErrorInvalidValue;

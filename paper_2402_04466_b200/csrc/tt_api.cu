@@ -664,6 +664,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
       const int bns[3] = {64, 128, 256};
       q.block_n = bns[bi]; q.map_b = L.map_b[bi]; q.n_tiles_n = L.cout / q.block_n;
       q.cout = L.cout; q.bias = L.b; q.status = ctx->status_dev;
+      q.n_prod = 3;
       return TT_OK;
     };
     for (int l = 1; l < ctx->n_enc; ++l) {
@@ -694,7 +695,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
   po.head_w = ctx->head_w; po.head_b = ctx->head_b; po.conf_w = ctx->conf_w; po.conf_b = ctx->conf_b;
   po.conf_mode = c.conf_mode; po.zthr = ctx->zthr;
   po.logits = ctx->logits; po.probs = ctx->probs; po.masks = ctx->masks; po.bits = ctx->bits;
-  po.results = ctx->results_dev; po.scratch = ctx->post_scratch;
+  po.results = ctx->results_dev; po.scratch = ctx->post_scratch; po.status = ctx->status_dev;
   TT_CUDA(ctx, launch_postprocess(po, s));
   if ((ms_ = mark_stage(ctx, TT_STAGE_POSTPROCESS, 2)) != TT_OK) return ms_;
 

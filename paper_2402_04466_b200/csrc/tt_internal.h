@@ -97,6 +97,7 @@ struct ConvTcParams {
   int32_t tiles_x, tiles_y; // 16 x 8 pixel patches
   int32_t n_tiles_n;        // CoutPacked / block_n
   int32_t block_n;          // 64, 128 or 256
+  int32_t n_prod;           // producer warps that issue loads, 1..3
   int32_t cout;             // real output channels (RELU) or 4*hidden (LSTM)
   int32_t epilogue;
   const float* bias;        // packed order, [CoutPacked]
@@ -132,6 +133,7 @@ struct PostParams {
   uint8_t* bits;        // optional [K][plane], bit t = mask of tool t
   tt_result* results;   // device, [K]
   void* scratch;
+  int32_t* status;      // optional device word: set non-zero when a bounded wait ran out
 };
 size_t post_scratch_bytes(int K, int hm, int wm, int ch, int T);
 cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s);

@@ -62,6 +62,9 @@ def test_preprocess_fixed_points(cuda_device):
     ((3, 128, 60, 80, 7), "gap_linear"),      # endoscopy-scale grid
     ((1, 256, 23, 37, 7), "gap_linear"),      # odd plane, large hidden
     ((2, 64, 8, 8, 8), "mean_sigmoid"),       # exactly one tile, max tools
+    ((3, 512, 9, 11, 5), "gap_linear"),       # widest hidden state, plane not a multiple of 4
+    ((4, 128, 7, 5, 3), "mean_sigmoid"),      # fewer 4-pixel rounds than warps in the grid; ranges cross streams
+    ((8, 256, 31, 33, 8), "gap_linear"),      # 8 streams, max tools, ragged plane
 ])
 def test_postprocess_matches_oracle(cuda_device, channels_last, shape, conf_mode):
     K, ch, hm, wm, T = shape
