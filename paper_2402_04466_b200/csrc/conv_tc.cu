@@ -162,7 +162,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
       const int m = tile / p.n_tiles_n;
       const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
       const int x0 = tx * PATCH_W, y0 = ty * PATCH_H;
-      const int img_a[2] = {s_img[img], s_img[TT_MAX_STREAMS + img]};
+      // (two scalars, not an indexed array: an array would live in local memory, and a memory round
+      // trip in this thread's loop delays every copy it issues)
+      const int img_x = s_img[img], img_h = s_img[TT_MAX_STREAMS + img];
       for (; it < k_iters; it += n_prod) {
         const int4 e = s_tab[it];
         ok = mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag, p.status, 0x100 + (int)stage);
@@ -170,7 +172,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
         const uint32_t fb = smem_u32(full_bar + stage);
         uint8_t* st = smem + stage * Cfg::STAGE_BYTES;
         mbar_arrive_expect_tx(fb, Cfg::STAGE_BYTES);
-        tma_load_4d(smem_u32(st), maps + e.x * (int)sizeof(TensorMap128), fb, e.y, x0 + e.z, y0 + e.w, img_a[e.x >> 2]);
+        tma_load_4d(smem_u32(st), maps + e.x * (int)sizeof(TensorMap128), fb, e.y, x0 + e.z, y0 + e.w, e.x < 4 ? img_x : img_h);
         tma_load_2d(smem_u32(st + Cfg::A_BYTES), &p.map_b, fb, it * SLAB_C, nt * BLOCK_N);
         stage += (uint32_t)n_prod;
         if (stage >= (uint32_t)STAGES) { stage -= STAGES; phase ^= 1u; }
@@ -179,29 +181,34 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     }
   } else if (warp == MMA_WARP && lane == 0) {
     // -------------------------------------------------------------------- MMA issuer
+    // This loop is one thread's chain of dependent instructions and sets the pace of the whole
+    // block, so everything that does not change is formed once: the operand descriptors differ
+    // between stages only in their 14-bit address field (16-byte units; shared memory is far
+    // below the field's range, so plain additions never carry out of it).
     uint32_t stage = 0, phase = 0, acc_phase = 0;
     int acc = 0;
     bool ok = true;
+    const uint64_t a_desc0 = make_smem_desc(smem_u32(smem), SBO, LAYOUT);
+    constexpr uint64_t STAGE_UNITS = Cfg::STAGE_BYTES >> 4, B_UNITS = Cfg::A_BYTES >> 4;
+    const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
+    uint64_t a_desc = a_desc0;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       ok = mbar_wait(smem_u32(tempty_bar + acc), acc_phase ^ 1u, abort_flag, p.status, 0x200 + acc);
       if (!ok) break;
-      tc_fence_after();
+      tc_fence_after();   // the epilogue's TMEM reads of this buffer come before the MMAs that overwrite it
       const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BLOCK_N);
       for (int it = 0; it < k_iters; ++it) {
-        ok = mbar_wait(smem_u32(full_bar + stage), phase, abort_flag, p.status, 0x300 + (int)stage);
+        // the copies complete on the barrier through the async proxy, which the MMAs read through too
+        ok = mbar_wait(full0 + 8u * stage, phase, abort_flag, p.status, 0x300 + (int)stage);
         if (!ok) break;
-        tc_fence_after();
-        const uint32_t a_addr = smem_u32(smem + stage * Cfg::STAGE_BYTES);
-        const uint32_t b_addr = a_addr + Cfg::A_BYTES;
-        const uint64_t a_desc = make_smem_desc(a_addr, SBO, LAYOUT);
-        const uint64_t b_desc = make_smem_desc(b_addr, SBO, LAYOUT);
+        const uint64_t b_desc = a_desc + B_UNITS;
+        // advance along K inside the swizzle atom: 16 bf16 = 32 bytes = 2 descriptor units
+        umma_bf16(d_tmem, a_desc, b_desc, IDESC, it != 0 ? 1u : 0u);
 #pragma unroll
-        for (int k = 0; k < SLAB_C / UMMA_K; ++k) {
-          // advance along K inside the swizzle atom: 16 bf16 = 32 bytes = 2 descriptor units
-          umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), IDESC, (it | k) != 0 ? 1u : 0u);
-        }
-        umma_commit(smem_u32(empty_bar + stage));  // frees the stage once the MMAs have read it
-        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        for (int k = 1; k < SLAB_C / UMMA_K; ++k) umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), IDESC, 1u);
+        umma_commit(empty0 + 8u * stage);            // frees the stage once the MMAs have read it
+        a_desc += STAGE_UNITS;
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; a_desc = a_desc0; }
       }
       if (!ok) break;
       umma_commit(smem_u32(tfull_bar + acc));      // accumulator complete

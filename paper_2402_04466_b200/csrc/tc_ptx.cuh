@@ -10,6 +10,10 @@ namespace tt {
 namespace tc {
 
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // about 2 s of SM cycles per wait
+// How long one try_wait may keep its thread suspended inside the barrier unit before it reports
+// "not yet": a suspended thread issues nothing, a thread that polls in a loop takes issue slots
+// from the warps that share its scheduler.
+constexpr uint32_t TRY_WAIT_SUSPEND_NS = 20000u;
 
 // ------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -21,10 +25,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(TRY_WAIT_SUSPEND_NS)
       : "memory");
   return ok != 0;
 }

@@ -4,6 +4,7 @@
 #include <cuda.h>
 
 #include <chrono>
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -353,7 +354,10 @@ int pick_block_n(const TcLayer& L, int m_tiles, int sm_count) {
     if (!L.has_b[i]) continue;
     const long tiles = (long)m_tiles * (L.cout / bns[i]);
     const long waves = (tiles + sm_count - 1) / sm_count;
-    const double cost = (double)waves * (bns[i] + 48);
+    // Time of a tile: its main loop is paced by the thread that issues the MMAs (about 600 cycles
+    // per K slab whatever the width) until the tensor pipe itself needs longer (2 cycles per
+    // column and K slab of 64 at 128 rows).
+    const double cost = (double)waves * std::max(600.0, 2.5 * bns[i]);
     if (best < 0 || cost < best_cost - 1e-9 || (std::fabs(cost - best_cost) < 1e-9 && bns[i] > bns[best])) {
       best = i;
       best_cost = cost;
