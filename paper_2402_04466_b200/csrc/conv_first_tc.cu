@@ -2,11 +2,13 @@
 // preprocess) -> COUT channels, 3x3, pad 1, stride 1 or 2, bias, ReLU, output bf16 channels-last.
 //
 // K = 27 (padded to 32) makes the arithmetic free on tcgen05; the layer is then bound by HBM
-// (read the fp32 input once, write the bf16 output once).  The A operand cannot come from TMA
-// (planar fp32 source, 3 channels), so four producer warps build it: they first copy the input
-// patch of the tile (all three planes, with halo, zero-filled outside the image) into shared
-// memory with coalesced loads -- the loads of the next tile are already in flight while the
-// current one is being used -- then each thread picks the 27 taps of one output pixel from
+// (read the fp32 input once, write the bf16 output once).  The A operand cannot come straight
+// from TMA (planar fp32 source, 3 channels), so four producer warps build it.  The input patch of
+// a tile (all three planes, with halo) arrives in shared memory as one TMA box load; the box starts
+// three columns left of the halo so that its first byte is 16-byte aligned, and everything outside
+// the image is zero-filled by the TMA unit, which is the convolution's padding.  Two patch buffers
+// keep the loads of the next two tiles in flight while the current one is used.  Each producer
+// thread picks the 27 taps of one output pixel from
 // shared memory, rounds them to bf16 and writes one 64-byte row of the
 // [128 pixels][32] operand tile in the no-swizzle K-major core-matrix layout (8 rows x 16 bytes
 // contiguous; neighbouring core matrices 128 bytes apart along K, 512 bytes apart along M).
@@ -28,23 +30,29 @@ constexpr int F_A_BYTES = 128 * 64;                 // 128 rows x 32 bf16
 constexpr int F_THREADS = 288;                      // warps 0-3 gather, 4 MMA, 5-8 epilogue
 constexpr int F_TMEM_COLS = 128;                    // two accumulator buffers of up to 64 columns
 
+// Columns of the input patch box: 3 columns in front for alignment, the 15*stride + 3 columns of
+// the patch, rounded up to a multiple of 4 (16 bytes).
+__host__ __device__ constexpr int box_w(int stride) { return (15 * stride + 3 + 3 + 3) & ~3; }
+
 template <int COUT, int STRIDE>
 __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
   constexpr int PH = 7 * STRIDE + 3, PW = 15 * STRIDE + 3;   // input patch of a 16 x 8 output tile
-  constexpr int PATCH = 3 * PH * PW;
-  constexpr int NPF = (PATCH + 127) / 128;                   // patch elements per producer thread
+  constexpr int BW = box_w(STRIDE);                          // box columns: 3 alignment columns + PW, rounded up to 4
+  constexpr int PATCH_BYTES = 3 * PH * BW * 4;
+  constexpr int PATCH_STRIDE = (PATCH_BYTES + 127) & ~127;   // patch buffers stay 128-byte aligned
   extern __shared__ uint8_t smem_raw[];
   uint8_t* s_out = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);  // one output tile, TMA box layout
   uint8_t* s_a = s_out + 128 * COUT * 2;                      // operand ring
   uint8_t* s_b = s_a + F_STAGES * F_A_BYTES;                  // weights in operand layout
-  float (*s_patch)[PATCH] = reinterpret_cast<float (*)[PATCH]>(s_b + COUT * 64);  // [2][PATCH]
-  __shared__ __align__(8) uint64_t s_bar[2 * F_STAGES + 4];
+  uint8_t* s_patch = s_b + COUT * 64;                         // [2] patches of [3][PH][BW] floats
+  __shared__ __align__(8) uint64_t s_bar[2 * F_STAGES + 6];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   uint64_t* a_full = s_bar;                 // [F_STAGES] 128 gather threads arrive
   uint64_t* a_empty = s_bar + F_STAGES;     // [F_STAGES] MMA commit
   uint64_t* t_full = s_bar + 2 * F_STAGES;  // [2] MMA commit
   uint64_t* t_empty = t_full + 2;           // [2] 4 epilogue warps arrive
+  uint64_t* p_full = t_empty + 2;           // [2] patch landed (TMA transaction bytes)
   volatile int* abort_flag = &s_abort;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -56,6 +64,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(t_full + a), 1);
       mbar_init(smem_u32(t_empty + a), 4);
+      mbar_init(smem_u32(p_full + a), 1);
     }
     s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -77,7 +86,6 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
 
   const int tiles_per_img = p.tiles_x * p.tiles_y;
   const int total_tiles = p.K * tiles_per_img;
-  const size_t in_plane = (size_t)p.H * p.W;
 
   if (warp < 4) {
     // ------------------------------------------------------------------ operand producers
@@ -85,36 +93,26 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
     const int row = ptid;
     const int py = row >> 4, px = row & 15;
     uint8_t* my_row = s_a + (row >> 3) * 512 + (row & 7) * 16;   // + kc * 128 per 16-byte chunk
-    uint32_t stage = 0, phase = 0;
+    uint32_t stage = 0, phase = 0, pphase = 0;
     int buf = 0;
-    float pf[NPF];
 
-    // coalesced fetch of one tile's input patch into registers (zero outside the image)
-    auto fetch_patch = [&](int tile) {
+    // one thread starts the box load of a tile's input patch into patch buffer b
+    auto fetch_patch = [&](int tile, int b) {
       const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, img = tile / tiles_per_img;
-      const float* src = p.in + (size_t)img * 3 * in_plane;
-      const int x_in0 = tx * 16 * STRIDE - 1, y_in0 = ty * 8 * STRIDE - 1;
-#pragma unroll
-      for (int i = 0; i < NPF; ++i) {
-        const int f = ptid + i * 128;
-        const int c = f / (PH * PW), r = (f / PW) % PH, col = f % PW;
-        const int yi = y_in0 + r, xi = x_in0 + col;
-        const bool ok = f < PATCH && yi >= 0 && yi < p.H && xi >= 0 && xi < p.W;
-        pf[i] = ok ? __ldg(src + (size_t)c * in_plane + (size_t)yi * p.W + xi) : 0.0f;
-      }
+      const uint32_t bar = smem_u32(p_full + b);
+      mbar_arrive_expect_tx(bar, PATCH_BYTES);
+      // column tx*16*STRIDE - 1 is the halo; the box starts 3 columns earlier, on a 16-byte boundary
+      tma_load_4d(smem_u32(s_patch + b * PATCH_STRIDE), &p.map_in, bar, tx * 16 * STRIDE - 4, ty * 8 * STRIDE - 1, 0, img);
     };
 
     bool fail = false;   // a bounded wait ran out; the four warps learn of it together at the barrier
-    if (blockIdx.x < total_tiles) fetch_patch(blockIdx.x);
+    if (ptid == 0) {
+      if (blockIdx.x < total_tiles) fetch_patch(blockIdx.x, 0);
+      if (blockIdx.x + gridDim.x < total_tiles) fetch_patch(blockIdx.x + gridDim.x, 1);
+    }
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-#pragma unroll
-      for (int i = 0; i < NPF; ++i) {
-        const int f = ptid + i * 128;
-        if (f < PATCH) s_patch[buf][f] = pf[i];
-      }
-      // the four producer warps meet here; with two patch buffers one barrier per tile is enough
-      if (named_barrier_or(1, 128, fail)) break;
-      if (tile + gridDim.x < total_tiles) fetch_patch(tile + gridDim.x);   // next tile's loads fly during the build
+      if (!fail && !mbar_wait(smem_u32(p_full + buf), pphase, abort_flag, p.status, 0x900 + buf)) fail = true;
+      const float* patch = reinterpret_cast<const float*>(s_patch + buf * PATCH_STRIDE);
       float v[27];
 #pragma unroll
       for (int c = 0; c < 3; ++c)
@@ -122,7 +120,14 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
         for (int ky = 0; ky < 3; ++ky)
 #pragma unroll
           for (int kx = 0; kx < 3; ++kx)
-            v[(c * 3 + ky) * 3 + kx] = s_patch[buf][(c * PH + py * STRIDE + ky) * PW + px * STRIDE + kx];
+            v[(c * 3 + ky) * 3 + kx] = patch[(c * PH + py * STRIDE + ky) * BW + px * STRIDE + kx + 3];
+      // the four producer warps meet here: everybody has read this patch buffer, it can be refilled
+      if (named_barrier_or(1, 128, fail)) break;
+      if (ptid == 0 && tile + 2 * (int)gridDim.x < total_tiles) {
+        fence_proxy_async_smem();
+        fetch_patch(tile + 2 * gridDim.x, buf);
+      }
+      if (buf) pphase ^= 1u;
       buf ^= 1;
       if (!mbar_wait(smem_u32(a_empty + stage), phase ^ 1u, abort_flag, p.status, 0x500 + (int)stage)) {
         fail = true;
@@ -233,8 +238,8 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
 
 template <int COUT, int STRIDE>
 cudaError_t launch_t(const ConvFirstTcParams& p, int grid, cudaStream_t s) {
-  constexpr int PH = 7 * STRIDE + 3, PW = 15 * STRIDE + 3;
-  constexpr int SMEM = 1024 + 128 * COUT * 2 + F_STAGES * F_A_BYTES + COUT * 64 + 2 * 3 * PH * PW * 4;
+  constexpr int PH = 7 * STRIDE + 3;
+  constexpr int SMEM = 1024 + 128 * COUT * 2 + F_STAGES * F_A_BYTES + COUT * 64 + 2 * ((3 * PH * box_w(STRIDE) * 4 + 127) & ~127);
   auto kern = conv_first_tc_kernel<COUT, STRIDE>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
@@ -245,6 +250,7 @@ cudaError_t launch_t(const ConvFirstTcParams& p, int grid, cudaStream_t s) {
 }  // namespace
 
 bool conv_first_tc_supported(int cout) { return cout == 32 || cout == 64; }
+int conv_first_tc_box_w(int stride) { return box_w(stride); }
 
 // [cout][27] bf16 bit patterns (row-major, k = c*9 + ky*3 + kx) -> operand layout, cout*32 values
 void conv_first_tc_pack(const uint16_t* w_bf16, int cout, uint16_t* packed) {

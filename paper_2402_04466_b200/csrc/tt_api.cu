@@ -284,6 +284,19 @@ tt_status encode_map(tt_ctx* ctx, TensorMap128* out, void* base, int rank, const
   return TT_OK;
 }
 
+// Plain (unswizzled) map of an fp32 tensor.
+tt_status encode_map_f32(tt_ctx* ctx, TensorMap128* out, void* base, int rank, const cuuint64_t* dims,
+                         const cuuint64_t* strides_bytes, const cuuint32_t* box) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return fail(ctx, TT_ERR_CUDA, "cuTensorMapEncodeTiled entry point unavailable");
+  cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+  CUresult r = fn(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, base, dims,
+                  strides_bytes, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ctx, TT_ERR_CUDA, "cuTensorMapEncodeTiled (fp32) failed with code %d", (int)r);
+  return TT_OK;
+}
+
 // Activation maps for one NHWC bf16 source [n_img][H][W][C] consumed at the given stride.
 // stride 1: one map (index 0).  stride 2: four parity views, index ypar*2 + xpar.
 tt_status make_act_maps(tt_ctx* ctx, TensorMap128* maps4, __nv_bfloat16* base, int n_img, int H, int W, int C,
@@ -508,7 +521,8 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
       return st;
   } else {
     if (ctx->lay_c[1] % 8) return fail(ctx, TT_ERR_UNSUPPORTED, "bf16 path needs enc_cout[0] in multiples of 8");
-    if (conv_first_tc_supported(ctx->lay_c[1])) {
+    // the tensor-core first layer fetches its input patches with TMA: rows of the planar fp32 input must be 16-byte multiples
+    if (conv_first_tc_supported(ctx->lay_c[1]) && c.net_w % 4 == 0 && (c.enc_stride[0] == 1 || c.enc_stride[0] == 2)) {
       const int co = ctx->lay_c[1];
       std::vector<uint16_t> wb((size_t)co * 27), packed((size_t)co * 32);
       for (size_t i = 0; i < wb.size(); ++i) wb[i] = f32_to_bf16_rne(w->enc_w[0][i]);
@@ -528,6 +542,12 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
         const cuuint64_t str[3] = {(cuuint64_t)co * 2, (cuuint64_t)f.Wo * co * 2, (cuuint64_t)f.Ho * f.Wo * co * 2};
         const cuuint32_t box[4] = {(cuuint32_t)co, 16, 8, 1};
         if ((st = encode_map(ctx, &f.map_out, ctx->enc_out[0], 4, dims, str, box, co * 2)) != TT_OK) return st;
+      }
+      {
+        const cuuint64_t dims[4] = {(cuuint64_t)f.W, (cuuint64_t)f.H, 3, (cuuint64_t)S};
+        const cuuint64_t str[3] = {(cuuint64_t)f.W * 4, (cuuint64_t)f.H * f.W * 4, (cuuint64_t)3 * f.H * f.W * 4};
+        const cuuint32_t box[4] = {(cuuint32_t)conv_first_tc_box_w(f.stride), (cuuint32_t)(7 * f.stride + 3), 3, 1};
+        if ((st = encode_map_f32(ctx, &f.map_in, ctx->pre, 4, dims, str, box)) != TT_OK) return st;
       }
       ctx->use_first_tc = true;
     } else if ((st = pack_simt(ctx, &ctx->simt_enc[0], w->enc_w[0], w->enc_b[0], 3, ctx->lay_c[1], c.enc_stride[0],

@@ -66,6 +66,7 @@ struct alignas(64) TensorMap128 {
 // On the tensor cores (cout 32 or 64): operand tiles are built by producer threads.
 struct ConvFirstTcParams {
   TensorMap128 map_out;       // output [K][Ho][Wo][cout] bf16, box [cout][16][8][1], 128B / 64B swizzle
+  TensorMap128 map_in;        // input [K][3][H][W] fp32, box [conv_first_tc_box_w(stride)][7*stride+3][3][1], no swizzle
   const float* in;            // [K][3][H][W] fp32
   __nv_bfloat16* out;         // [K][Ho][Wo][cout] bf16
   int32_t H, W, Ho, Wo, stride, K, cout, tiles_x, tiles_y;
@@ -74,6 +75,7 @@ struct ConvFirstTcParams {
   int32_t* status;
 };
 bool conv_first_tc_supported(int cout);
+int conv_first_tc_box_w(int stride);   // columns of the input patch box (a multiple of 4)
 void conv_first_tc_pack(const uint16_t* w_bf16, int cout, uint16_t* packed);
 cudaError_t launch_conv_first_tc(const ConvFirstTcParams& p, int sm_count, cudaStream_t s);
 
