@@ -245,8 +245,11 @@ __global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const __grid_co
 // that does not depend on how the work is divided (the pooled state per unit, probabilities per
 // pixel), so a stream's results are bit for bit the same whatever else shares the launch.
 constexpr int SW_ROUND_PIX = 4;
-constexpr int SW_UNIT_ROUNDS = 8;           // rounds per unit
-constexpr int SW_UNIT_PIX = SW_ROUND_PIX * SW_UNIT_ROUNDS;
+// Rounds per unit: 8 (32 pixels, whole 128-byte lines per store) on large maps; 2 on small ones,
+// where a launch has so few units that the time of one warp's unit sets the kernel's duration.
+// A function of the map size alone, so that a stream's sums are grouped the same way whatever
+// else shares the launch.
+__host__ __device__ inline int sw_unit_rounds(int plane) { return plane >= 8192 ? 8 : 2; }
 constexpr int SW_OUT_ROW = 36;              // floats per tool row of the parked logits: (4*t + pixel) % 32 is conflict-free
 constexpr int SW_OUT_FLOATS = TT_MAX_TOOLS * SW_OUT_ROW;
 constexpr long long SW_WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s of SM cycles
@@ -362,7 +365,8 @@ __global__ void __launch_bounds__(StreamCfg<NCHUNK>::THREADS, 1) post_stream_ker
   const int T = p.T;
   const int plane = p.Hm * p.Wm;
   const int rpi = (plane + SW_ROUND_PIX - 1) / SW_ROUND_PIX;    // rounds per image
-  const int upi = (plane + SW_UNIT_PIX - 1) / SW_UNIT_PIX;      // units per image
+  const int unit_rounds = sw_unit_rounds(plane), unit_pix = unit_rounds * SW_ROUND_PIX;
+  const int upi = (plane + unit_pix - 1) / unit_pix;            // units per image
   const int total_units = p.K * upi;
   const int u_begin = (int)((long long)blockIdx.x * total_units / gridDim.x);
   const int u_end = (int)((long long)(blockIdx.x + 1) * total_units / gridDim.x);
@@ -394,7 +398,7 @@ __global__ void __launch_bounds__(StreamCfg<NCHUNK>::THREADS, 1) post_stream_ker
 
   if (u_begin + warp < u_end) {
     // lane 0: the next round to copy (unit, stream, first pixel, rounds left in the unit)
-    int iss_unit = u_begin + warp, iss_n = iss_unit / upi, iss_pix = (iss_unit % upi) * SW_UNIT_PIX, iss_stage = 0;
+    int iss_unit = u_begin + warp, iss_n = iss_unit / upi, iss_pix = (iss_unit % upi) * unit_pix, iss_stage = 0;
     auto issue = [&]() {
       const int npix = min(SW_ROUND_PIX, plane - iss_pix);
       const uint32_t bytes = (uint32_t)npix * CH * 4u;
@@ -406,10 +410,10 @@ __global__ void __launch_bounds__(StreamCfg<NCHUNK>::THREADS, 1) post_stream_ker
                    ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
       if (++iss_stage == STAGES) iss_stage = 0;
       iss_pix += SW_ROUND_PIX;
-      if ((iss_pix & (SW_UNIT_PIX - 1)) == 0 || iss_pix >= plane) {   // unit exhausted: on to this warp's next one
+      if ((iss_pix & (unit_pix - 1)) == 0 || iss_pix >= plane) {   // unit exhausted: on to this warp's next one
         iss_unit += SW_WARPS;
         iss_n = iss_unit / upi;
-        iss_pix = (iss_unit % upi) * SW_UNIT_PIX;
+        iss_pix = (iss_unit % upi) * unit_pix;
       }
     };
     if (lane == 0)
@@ -426,11 +430,11 @@ __global__ void __launch_bounds__(StreamCfg<NCHUNK>::THREADS, 1) post_stream_ker
     long long spf = 0;                               // lane t < T: sum of tool t's probabilities, fixed point
     int stream_rounds = 0;                           // rounds of the current stream done by this warp
 
-    // write out the parked logits of one unit of stream n (pixels pix0 .. pix0+31); lane = pixel
-    auto write_unit = [&](int n, int pix0) {
+    // write out the parked logits of one unit of stream n (pixels pix0 .. pix0 + 4*rounds - 1); lane = pixel
+    auto write_unit = [&](int n, int pix0, int rounds) {
       __syncwarp();
       const int pix = pix0 + lane;
-      const bool live = pix < plane;
+      const bool live = lane < rounds * SW_ROUND_PIX && pix < plane;
       const int px = live ? pix % p.Wm : 0, py = live ? pix / p.Wm : 0;
       uint32_t bits = 0;
 #pragma unroll
@@ -521,8 +525,8 @@ __global__ void __launch_bounds__(StreamCfg<NCHUNK>::THREADS, 1) post_stream_ker
 #pragma unroll 1
     for (int unit = u_begin + warp; unit < u_end && ok; unit += SW_WARPS) {
       const int n = unit / upi;
-      const int unit_pix0 = (unit % upi) * SW_UNIT_PIX;
-      const int rounds = min(SW_UNIT_ROUNDS, (plane - unit_pix0 + SW_ROUND_PIX - 1) / SW_ROUND_PIX);
+      const int unit_pix0 = (unit % upi) * unit_pix;
+      const int rounds = min(unit_rounds, (plane - unit_pix0 + SW_ROUND_PIX - 1) / SW_ROUND_PIX);
       if (n != cur_n) {                              // this warp's units run on into the next stream
         flush_stream(cur_n);
         cur_n = n;
@@ -612,7 +616,7 @@ __global__ void __launch_bounds__(StreamCfg<NCHUNK>::THREADS, 1) post_stream_ker
 #pragma unroll
         for (int i = 0; i < NCHUNK * 4; ++i) gap[i] += to_fixed(gsum[i]);
       }
-      write_unit(n, unit_pix0);
+      write_unit(n, unit_pix0, rounds);
     }
     if (ok && stream_rounds) flush_stream(cur_n);
   }
@@ -746,7 +750,8 @@ cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s) {
     cudaError_t e = post_sm_count(&sms);
     if (e != cudaSuccess) return e;
     // persistent: one block per multiprocessor, fewer when there is less than a unit per warp
-    const long long units = (long long)p.K * ((plane + SW_UNIT_PIX - 1) / SW_UNIT_PIX);
+    const int unit_pix = sw_unit_rounds(plane) * SW_ROUND_PIX;
+    const long long units = (long long)p.K * ((plane + unit_pix - 1) / unit_pix);
     const int warps = p.Ch == 512 ? StreamCfg<4>::WARPS : StreamCfg<1>::WARPS;
     const long long want = (units + warps - 1) / warps;
     const int grid = (int)(want < sms ? want : sms);

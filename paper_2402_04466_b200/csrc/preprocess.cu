@@ -135,18 +135,31 @@ preprocess_staged_kernel(const __grid_constant__ PreprocessParams p, int row_cap
     const int base0 = (y0 - sy_lo) * row_cap_bytes + (int)((src_lo + (uint32_t)(y0 * p.src_pitch + 3 * sx_lo)) & 15u);
     const int base1 = (y1 - sy_lo) * row_cap_bytes + (int)((src_lo + (uint32_t)(y1 * p.src_pitch + 3 * sx_lo)) & 15u);
     float o0[4], o1[4], o2[4];  // the three channels of the 4 outputs
+    if (fy == 0.0f) {
+      // The sample sits exactly on a source row (every row of an axis that is not resized): the
+      // lower row has weight zero, so top + 0 * (bot - top) = top and only one row is fetched.
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint32_t lo0, hi0, lo1, hi1;
-      fetch_pair(s_words, base0 + xoffs[j], lo0, hi0);
-      fetch_pair(s_words, base1 + xoffs[j], lo1, hi1);
-      // channel c of the left pixel is byte c of lo; of the right pixel: byte 3 of lo, bytes 0, 1 of hi
-      o0[j] = blend_magic(byte_to_magic(lo0, 0x7440), byte_to_magic(lo0, 0x7443), byte_to_magic(lo1, 0x7440),
-                          byte_to_magic(lo1, 0x7443), fxs[j], fy, scale, shift);
-      o1[j] = blend_magic(byte_to_magic(lo0, 0x7441), byte_to_magic(hi0, 0x7440), byte_to_magic(lo1, 0x7441),
-                          byte_to_magic(hi1, 0x7440), fxs[j], fy, scale, shift);
-      o2[j] = blend_magic(byte_to_magic(lo0, 0x7442), byte_to_magic(hi0, 0x7441), byte_to_magic(lo1, 0x7442),
-                          byte_to_magic(hi1, 0x7441), fxs[j], fy, scale, shift);
+      for (int j = 0; j < 4; ++j) {
+        uint32_t lo0, hi0;
+        fetch_pair(s_words, base0 + xoffs[j], lo0, hi0);
+        o0[j] = fmaf(fmaf(fxs[j], byte_to_magic(lo0, 0x7443) - byte_to_magic(lo0, 0x7440), byte_to_magic(lo0, 0x7440) - 8388608.0f), scale, shift);
+        o1[j] = fmaf(fmaf(fxs[j], byte_to_magic(hi0, 0x7440) - byte_to_magic(lo0, 0x7441), byte_to_magic(lo0, 0x7441) - 8388608.0f), scale, shift);
+        o2[j] = fmaf(fmaf(fxs[j], byte_to_magic(hi0, 0x7441) - byte_to_magic(lo0, 0x7442), byte_to_magic(lo0, 0x7442) - 8388608.0f), scale, shift);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        uint32_t lo0, hi0, lo1, hi1;
+        fetch_pair(s_words, base0 + xoffs[j], lo0, hi0);
+        fetch_pair(s_words, base1 + xoffs[j], lo1, hi1);
+        // channel c of the left pixel is byte c of lo; of the right pixel: byte 3 of lo, bytes 0, 1 of hi
+        o0[j] = blend_magic(byte_to_magic(lo0, 0x7440), byte_to_magic(lo0, 0x7443), byte_to_magic(lo1, 0x7440),
+                            byte_to_magic(lo1, 0x7443), fxs[j], fy, scale, shift);
+        o1[j] = blend_magic(byte_to_magic(lo0, 0x7441), byte_to_magic(hi0, 0x7440), byte_to_magic(lo1, 0x7441),
+                            byte_to_magic(hi1, 0x7440), fxs[j], fy, scale, shift);
+        o2[j] = blend_magic(byte_to_magic(lo0, 0x7442), byte_to_magic(hi0, 0x7441), byte_to_magic(lo1, 0x7442),
+                            byte_to_magic(hi1, 0x7441), fxs[j], fy, scale, shift);
+      }
     }
     float* d0 = p.dst + (size_t)n * 3 * plane + (size_t)yo * p.net_w + xo0;
     float* d1 = d0 + plane;
