@@ -36,8 +36,8 @@ __host__ __device__ constexpr int box_w(int stride) { return (15 * stride + 3 + 
 
 template <int COUT, int STRIDE>
 __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
-  constexpr int PH = 7 * STRIDE + 3, PW = 15 * STRIDE + 3;   // input patch of a 16 x 8 output tile
-  constexpr int BW = box_w(STRIDE);                          // box columns: 3 alignment columns + PW, rounded up to 4
+  constexpr int PH = 7 * STRIDE + 3;                         // rows of the input patch of a 16 x 8 output tile
+  constexpr int BW = box_w(STRIDE);                          // box columns: 3 alignment columns + the patch, rounded up to 4
   constexpr int PATCH_BYTES = 3 * PH * BW * 4;
   constexpr int PATCH_STRIDE = (PATCH_BYTES + 127) & ~127;   // patch buffers stay 128-byte aligned
   extern __shared__ uint8_t smem_raw[];
