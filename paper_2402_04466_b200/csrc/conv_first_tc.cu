@@ -55,6 +55,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
   uint64_t* p_full = t_empty + 2;           // [2] patch landed (TMA transaction bytes)
   volatile int* abort_flag = &s_abort;
 
+  pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < F_STAGES; ++s) {
@@ -83,6 +84,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = s_tmem;
+  pdl_wait();   // the set-up above read weights only; the input tensor is the previous kernel's output
 
   const int tiles_per_img = p.tiles_x * p.tiles_y;
   const int total_tiles = p.K * tiles_per_img;
@@ -243,8 +245,7 @@ cudaError_t launch_t(const ConvFirstTcParams& p, int grid, cudaStream_t s) {
   auto kern = conv_first_tc_kernel<COUT, STRIDE>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
-  kern<<<grid, F_THREADS, SMEM, s>>>(p);
-  return cudaGetLastError();
+  return launch_kernel(kern, grid, F_THREADS, SMEM, s, p, p.pdl != 0);
 }
 
 }  // namespace

@@ -88,6 +88,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
   int4* s_tab = reinterpret_cast<int4*>(bar_mem + Cfg::BAR_BYTES);            // [k_iters] {map slot, channel offset, dx, dy}
   int* s_img = reinterpret_cast<int*>(s_tab + MAX_K_ITERS);                   // [4][TT_MAX_STREAMS]: img0, img1, c_idx, h_out_idx
 
+  pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_per_img = p.tiles_x * p.tiles_y;
   const int total_tiles = p.K * tiles_per_img * p.n_tiles_n;
@@ -146,6 +147,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();   // everything above touched no activation; from here on the previous kernel's outputs are read
 
   const int n_prod = p.n_prod;
   const int prod = warp == 0 ? 0 : warp - (EPI_WARP0 + EPI_WARPS) + 1;   // producer index of warps 0, 10, 11
@@ -339,8 +341,7 @@ cudaError_t launch_cfg(const ConvTcParams& p, int sm_count, cudaStream_t s) {
   if (e != cudaSuccess) return e;
   const int total_tiles = p.K * p.tiles_x * p.tiles_y * p.n_tiles_n;
   const int grid = total_tiles < sm_count ? total_tiles : sm_count;
-  kern<<<grid, TC_THREADS, Cfg::SMEM_BYTES, s>>>(p);
-  return cudaGetLastError();
+  return launch_kernel(kern, grid, TC_THREADS, Cfg::SMEM_BYTES, s, p, p.pdl != 0);
 }
 
 template <int EPI>

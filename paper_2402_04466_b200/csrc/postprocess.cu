@@ -343,6 +343,7 @@ __device__ __forceinline__ void finish_stream_warp(const PostParams& p, int n, l
 
 template <int NCHUNK>
 __global__ void __launch_bounds__(StreamCfg<NCHUNK>::THREADS, 1) post_stream_kernel(const __grid_constant__ PostParams p) {
+  pdl_launch_dependents();
   using Cfg = StreamCfg<NCHUNK>;
   constexpr int CH = Cfg::CH;
   constexpr int STAGES = Cfg::STAGES;
@@ -392,6 +393,7 @@ __global__ void __launch_bounds__(StreamCfg<NCHUNK>::THREADS, 1) post_stream_ker
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  pdl_wait();   // head weights and barriers are set up; the hidden state is the previous kernel's output
 
   const ScratchLayout sl = scratch_layout(p.K, plane, CH, T);
   uint8_t* scr = reinterpret_cast<uint8_t*>(p.scratch);
@@ -755,9 +757,10 @@ cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s) {
     const int warps = p.Ch == 512 ? StreamCfg<4>::WARPS : StreamCfg<1>::WARPS;
     const long long want = (units + warps - 1) / warps;
     const int grid = (int)(want < sms ? want : sms);
-    if (p.Ch == 128) post_stream_kernel<1><<<grid, StreamCfg<1>::THREADS, StreamCfg<1>::SMEM_BYTES, s>>>(p);
-    else if (p.Ch == 256) post_stream_kernel<2><<<grid, StreamCfg<2>::THREADS, StreamCfg<2>::SMEM_BYTES, s>>>(p);
-    else post_stream_kernel<4><<<grid, StreamCfg<4>::THREADS, StreamCfg<4>::SMEM_BYTES, s>>>(p);
+    const bool pdl = p.pdl != 0;
+    if (p.Ch == 128) return launch_kernel(post_stream_kernel<1>, grid, StreamCfg<1>::THREADS, StreamCfg<1>::SMEM_BYTES, s, p, pdl);
+    if (p.Ch == 256) return launch_kernel(post_stream_kernel<2>, grid, StreamCfg<2>::THREADS, StreamCfg<2>::SMEM_BYTES, s, p, pdl);
+    return launch_kernel(post_stream_kernel<4>, grid, StreamCfg<4>::THREADS, StreamCfg<4>::SMEM_BYTES, s, p, pdl);
   } else {
     post_tile_kernel<<<p.K * nb, POST_THREADS, post_smem_bytes(p.Ch), s>>>(p);
   }

@@ -666,6 +666,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
   } else {
     if (ctx->use_first_tc) {
       ctx->first_tc.K = K;
+      ctx->first_tc.pdl = ctx->profiling ? 0 : 1;
       TT_CUDA(ctx, launch_conv_first_tc(ctx->first_tc, ctx->sm_count, s));
       if ((ms_ = mark_stage(ctx, TT_STAGE_ENC0, 1)) != TT_OK) return ms_;
     } else {
@@ -689,6 +690,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
       q.block_n = bns[bi]; q.map_b = L.map_b[bi]; q.n_tiles_n = L.cout / q.block_n;
       q.cout = L.cout; q.bias = L.b; q.status = ctx->status_dev;
       q.n_prod = 3;
+      q.pdl = ctx->profiling ? 0 : 1;
       return TT_OK;
     };
     for (int l = 1; l < ctx->n_enc; ++l) {
@@ -720,6 +722,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
   po.conf_mode = c.conf_mode; po.zthr = ctx->zthr;
   po.logits = ctx->logits; po.probs = ctx->probs; po.masks = ctx->masks; po.bits = ctx->bits;
   po.results = ctx->results_dev; po.scratch = ctx->post_scratch; po.status = ctx->status_dev;
+  po.pdl = (ctx->bf16 && !ctx->profiling) ? 1 : 0;
   TT_CUDA(ctx, launch_postprocess(po, s));
   if ((ms_ = mark_stage(ctx, TT_STAGE_POSTPROCESS, 2)) != TT_OK) return ms_;
 

@@ -9,6 +9,30 @@
 
 namespace tt {
 
+// Programmatic dependent launch.  A kernel launched with `pdl` set may start while its
+// predecessor in the stream is still running: its blocks take multiprocessors as the
+// predecessor's blocks leave them, do the set-up that touches no activation (barriers, tensor
+// memory, weight staging) and then wait in pdl_wait() until the predecessor has completed and its
+// writes are visible.  Without the launch attribute both device calls do nothing.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename Params>
+inline cudaError_t launch_kernel(void (*kern)(const Params), int grid, int block, size_t smem, cudaStream_t s, const Params& p,
+                                 bool pdl) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
 // Maps batch position n (0..K-1) of a launch to an image index inside a tensor that holds
 // more images than the batch (state slots, ping-pong halves).
 struct IdxMap {
@@ -70,6 +94,7 @@ struct ConvFirstTcParams {
   const float* in;            // [K][3][H][W] fp32
   __nv_bfloat16* out;         // [K][Ho][Wo][cout] bf16
   int32_t H, W, Ho, Wo, stride, K, cout, tiles_x, tiles_y;
+  int32_t pdl;                // launch as a programmatic dependent of the previous kernel in the stream
   const uint16_t* w_packed;   // device, cout*32 bf16 in the MMA operand layout
   const float* bias;          // device, [cout]
   int32_t* status;
@@ -100,6 +125,7 @@ struct ConvTcParams {
   int32_t n_tiles_n;        // CoutPacked / block_n
   int32_t block_n;          // 64, 128 or 256
   int32_t n_prod;           // producer warps that issue loads, 1..3
+  int32_t pdl;              // launch as a programmatic dependent of the previous kernel in the stream
   int32_t cout;             // real output channels (RELU) or 4*hidden (LSTM)
   int32_t epilogue;
   const float* bias;        // packed order, [CoutPacked]
@@ -136,6 +162,7 @@ struct PostParams {
   tt_result* results;   // device, [K]
   void* scratch;
   int32_t* status;      // optional device word: set non-zero when a bounded wait ran out
+  int32_t pdl;          // launch as a programmatic dependent of the previous kernel in the stream (channels-last kernel only)
 };
 size_t post_scratch_bytes(int K, int hm, int wm, int ch, int T);
 cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s);
