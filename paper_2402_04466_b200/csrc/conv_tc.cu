@@ -221,6 +221,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     constexpr int HALF_N = BLOCK_N / 2;           // columns handled by this warp
     constexpr int CHUNKS = HALF_N / 32;
     const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
+    // 32-byte stores of bf16 values need 16 values per pixel row between sector boundaries
+    const bool wide_out = EPI == TC_EPI_LSTM ? (p.hidden & 15) == 0 : (p.cout & 15) == 0;
     const int half = (warp - EPI_WARP0) >> 2;     // which half of the tile's columns
     const int row = quarter * 32 + lane;          // row of the 128-row tile = pixel of the patch
     const int py = row / PATCH_W, px = row % PATCH_W;
@@ -245,13 +247,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
         ho = ((size_t)s_img[3 * TT_MAX_STREAMS + img] * p.Ho * p.Wo + pix) * p.hidden + (col0 >> 2);
 #pragma unroll
         for (int ck = 0; ck < CHUNKS; ++ck) {
-          float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
-          if (valid && (col0 >> 2) + ck * 8 < p.hidden) {
-            lo = *reinterpret_cast<const float4*>(p.c_state + so + ck * 8);
-            hi = *reinterpret_cast<const float4*>(p.c_state + so + ck * 8 + 4);
-          }
-          c_old[ck * 8 + 0] = lo.x; c_old[ck * 8 + 1] = lo.y; c_old[ck * 8 + 2] = lo.z; c_old[ck * 8 + 3] = lo.w;
-          c_old[ck * 8 + 4] = hi.x; c_old[ck * 8 + 5] = hi.y; c_old[ck * 8 + 6] = hi.z; c_old[ck * 8 + 7] = hi.w;
+          float c8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          if (valid && (col0 >> 2) + ck * 8 < p.hidden) ld_global_v8(p.c_state + so + ck * 8, c8);
+#pragma unroll
+          for (int jj = 0; jj < 8; ++jj) c_old[ck * 8 + jj] = c8[jj];
         }
       }
 
@@ -259,6 +258,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
       if (!ok) break;
       tc_fence_after();
       const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N + half * HALF_N);
+      uint32_t hb[8];
 #pragma unroll
       for (int ck = 0; ck < CHUNKS; ++ck) {
         uint32_t v[32];
@@ -269,14 +269,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
             const float4* b4 = reinterpret_cast<const float4*>(p.bias + n0);
             __nv_bfloat16* dst = p.out + ((size_t)img * p.Ho * p.Wo + pix) * p.cout + n0;
 #pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              const float4 ba = __ldg(b4 + i / 4), bb = __ldg(b4 + i / 4 + 1);
-              uint4 u;
-              u.x = pack_bf16(fmaxf(__uint_as_float(v[i + 0]) + ba.x, 0.f), fmaxf(__uint_as_float(v[i + 1]) + ba.y, 0.f));
-              u.y = pack_bf16(fmaxf(__uint_as_float(v[i + 2]) + ba.z, 0.f), fmaxf(__uint_as_float(v[i + 3]) + ba.w, 0.f));
-              u.z = pack_bf16(fmaxf(__uint_as_float(v[i + 4]) + bb.x, 0.f), fmaxf(__uint_as_float(v[i + 5]) + bb.y, 0.f));
-              u.w = pack_bf16(fmaxf(__uint_as_float(v[i + 6]) + bb.z, 0.f), fmaxf(__uint_as_float(v[i + 7]) + bb.w, 0.f));
-              *reinterpret_cast<uint4*>(dst + i) = u;
+            for (int i = 0; i < 32; i += 16) {
+              uint32_t u[8];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float4 b = __ldg(b4 + i / 4 + j);
+                u[2 * j + 0] = pack_bf16(fmaxf(__uint_as_float(v[i + 4 * j + 0]) + b.x, 0.f), fmaxf(__uint_as_float(v[i + 4 * j + 1]) + b.y, 0.f));
+                u[2 * j + 1] = pack_bf16(fmaxf(__uint_as_float(v[i + 4 * j + 2]) + b.z, 0.f), fmaxf(__uint_as_float(v[i + 4 * j + 3]) + b.w, 0.f));
+              }
+              if (wide_out) {
+                st_global_v8_b32(dst + i, u);        // 16 channels = one 32-byte sector
+              } else {
+                *reinterpret_cast<uint4*>(dst + i) = make_uint4(u[0], u[1], u[2], u[3]);
+                *reinterpret_cast<uint4*>(dst + i + 8) = make_uint4(u[4], u[5], u[6], u[7]);
+              }
             }
           }
         } else {
@@ -294,18 +300,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
               c_new[jj] = fast_sigmoid(gf) * c_old[ck * 8 + jj] + fast_sigmoid(gi) * fast_tanh(gg);
               h_new[jj] = fast_sigmoid(go) * fast_tanh(c_new[jj]);
             }
-            float* c_ptr = p.c_state + so + ck * 8;
-            float* h_ptr = p.h_f32 + so + ck * 8;
-            *reinterpret_cast<float4*>(c_ptr) = make_float4(c_new[0], c_new[1], c_new[2], c_new[3]);
-            *reinterpret_cast<float4*>(c_ptr + 4) = make_float4(c_new[4], c_new[5], c_new[6], c_new[7]);
-            *reinterpret_cast<float4*>(h_ptr) = make_float4(h_new[0], h_new[1], h_new[2], h_new[3]);
-            *reinterpret_cast<float4*>(h_ptr + 4) = make_float4(h_new[4], h_new[5], h_new[6], h_new[7]);
-            uint4 hb;
-            hb.x = pack_bf16(h_new[0], h_new[1]);
-            hb.y = pack_bf16(h_new[2], h_new[3]);
-            hb.z = pack_bf16(h_new[4], h_new[5]);
-            hb.w = pack_bf16(h_new[6], h_new[7]);
-            *reinterpret_cast<uint4*>(p.h_bf16 + ho + ck * 8) = hb;
+            st_global_v8(p.c_state + so + ck * 8, c_new);
+            st_global_v8(p.h_f32 + so + ck * 8, h_new);
+            // bf16 shadow of h': 8 values are half a sector, so two neighbouring chunks leave together
+            const int hq = (ck & 1) * 4;
+            hb[hq + 0] = pack_bf16(h_new[0], h_new[1]);
+            hb[hq + 1] = pack_bf16(h_new[2], h_new[3]);
+            hb[hq + 2] = pack_bf16(h_new[4], h_new[5]);
+            hb[hq + 3] = pack_bf16(h_new[6], h_new[7]);
+            if (wide_out && CHUNKS % 2 == 0) {
+              if (ck & 1) st_global_v8_b32(p.h_bf16 + ho + (ck - 1) * 8, hb);
+            } else {
+              *reinterpret_cast<uint4*>(p.h_bf16 + ho + ck * 8) = make_uint4(hb[hq], hb[hq + 1], hb[hq + 2], hb[hq + 3]);
+            }
           }
         }
       }

@@ -331,6 +331,37 @@ def test_graph_replay_matches_plain_launches(cuda_device):
         assert np.array_equal(h1, h2) and np.array_equal(c1, c2)
 
 
+def test_dependent_launches_change_no_bit(cuda_device):
+    """The tensor-core kernels normally start as programmatic dependents of their predecessor (set-up overlapping
+    its tail); with stage profiling on every kernel is launched normally behind an event.  Both must give the same
+    bits, tick after tick, and stage times must come back in the profiled run."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="pdl", src_w=214, src_h=120, net_w=160, net_h=120, overlay=True)
+    K = 3
+    frames = _frames(wl, K, 4)
+    outs = []
+    for profiled in (False, True):
+        ctx, states, _ = _make(wl, K, overlay=True)
+        ctx.set_profiling(profiled)
+        per_tick = []
+        for t in range(4):
+            ctx.submit_frames([torch.from_numpy(frames[k][t]).to(cuda_device) for k in range(K)], states)
+            res = ctx.sync()
+            per_tick.append([(ctx.fetch_probs(r), ctx.fetch_masks(r), ctx.fetch_overlay(r), r["conf"].copy(), r["count"].copy())
+                             for r in res])
+        if profiled:
+            times = ctx.get_stage_times()
+            assert times["convlstm"] > 0 and times["postprocess"] > 0
+        outs.append((per_tick, [ctx.state_export(s) for s in states]))
+        ctx.destroy()
+    (a, ha), (b, hb) = outs
+    for ta, tb in zip(a, b):
+        for ra, rb in zip(ta, tb):
+            for va, vb in zip(ra, rb):
+                assert np.array_equal(va, vb)
+    for (h1, c1), (h2, c2) in zip(ha, hb):
+        assert np.array_equal(h1, h2) and np.array_equal(c1, c2)
+
+
 def test_two_submits_in_flight_match_serial_execution(cuda_device):
     """Software-pipelined use (submit t+1 before sync t, pinned host frames over the copy stream) must give
     bit for bit what one-at-a-time execution gives, with results returned oldest first."""
