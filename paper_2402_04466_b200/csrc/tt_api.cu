@@ -906,14 +906,15 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
   if (any_h2d) {
     TT_CUDA(ctx, cudaEventRecord(ctx->ev_copy, ctx->copy_stream));
     TT_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_copy, 0));
-    st = mark_stage(ctx, TT_STAGE_H2D, 0);
-    if (st != TT_OK) return st;
   }
   // frame pointers of this tick -> the slot's device table (the kernels read them from there)
   for (int n = 0; n < TT_MAX_STREAMS; ++n) ctx->frame_tab_host[slot][n] = n < K ? fp.p[n] : nullptr;
   TT_CUDA(ctx, cudaMemcpyAsync(ctx->frame_tab_dev[slot], ctx->frame_tab_host[slot], sizeof(void*) * TT_MAX_STREAMS,
                                cudaMemcpyHostToDevice, s));
   ctx->cur_tab = ctx->frame_tab_dev[slot];
+  // everything that moves host data to the device (frames, pointer table) counts as the H2D stage
+  st = mark_stage(ctx, TT_STAGE_H2D, 0);
+  if (st != TT_OK) return st;
 
   // The launch sequence of a tick is replayed from a CUDA graph once the same (K, slot, state
   // placement) has been seen before; the first occurrence runs as plain launches.  With stage
