@@ -229,8 +229,7 @@ __global__ void __launch_bounds__(POST_THREADS) post_tile_kernel(const __grid_co
 }
 
 // Channels-last fast path (hidden a multiple of 128): a persistent kernel of independent warps.
-// Every stream's pixels are cut into units of 32 consecutive pixels (8 rounds of 4; 8 pixels on
-// small maps, see sw_unit_rounds).  A block
+// Every stream's pixels are cut into units of 32 consecutive pixels (8 rounds of 4).  A block
 // takes a contiguous range of the (stream, unit) list and its warps take the units of that range
 // in turn (warp w: units w, w + WARPS, ...).  Each warp runs its own ring of bulk-copy stages:
 // lane 0 issues one cp.async.bulk per round (the round's 4 x CH floats are contiguous in memory)
