@@ -167,6 +167,23 @@ def test_bf16_odd_extents_on_strided_layers(cuda_device):
     _run_bf16(cuda_device, wl, 2, 3)
 
 
+def test_bf16_first_layer_patch_boxes_over_the_image_border(cuda_device):
+    """The tensor-core first layer fetches each tile's input patch as one TMA box whose start lies three columns
+    left of the halo; with a 148x110 input (rows are 16-byte multiples, nothing else is aligned) the boxes of the
+    right and bottom tiles reach past the image and the left and top ones start at negative coordinates."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="bf16-border", src_w=200, src_h=150, net_w=148, net_h=110,
+                                              enc_cout=(32, 64, 128), hidden=32)
+    assert wl.map_hw() == (14, 19)
+    _run_bf16(cuda_device, wl, 2, 3)
+
+
+def test_bf16_first_layer_stride1_on_the_tensor_cores(cuda_device):
+    """A stride-1 first layer (18-column patch, 24-column box) with an odd output height."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="bf16-first-s1", src_w=96, src_h=72, net_w=64, net_h=45,
+                                              enc_cout=(64, 64), enc_stride=(1, 2), hidden=32)
+    _run_bf16(cuda_device, wl, 2, 2)
+
+
 def test_bf16_first_layer_width_outside_the_tensor_core_kernel(cuda_device):
     """A first layer of 96 channels is not covered by the tensor-core first-layer kernel: the fp32 SIMT kernel writes
     the bf16 channels-last map instead, and the next layer runs on 32-channel slabs."""
