@@ -273,6 +273,19 @@ tt_status tt_set_profiling(tt_ctx* ctx, int32_t on);
 tt_status tt_get_stage_times(tt_ctx* ctx, float* ms);
 tt_status tt_get_counters(const tt_ctx* ctx, uint64_t* kernel_launches, uint64_t* ticks);
 
+/*
+ * tt_debug_expire_wait — failure-path probe, for tests.  Every barrier wait inside the kernels is
+ * bounded: when one runs out the kernel records a code in the context's status word and returns,
+ * and the tt_sync of that tick answers TT_ERR_DEVICE_STATUS (the paper's systems have no such
+ * path; it is this library's reading of "a failed client must not take the GPU down with it",
+ * Section IV-A).  This call enqueues, on the context's stream, one warp that waits through that
+ * same bounded wait on a barrier nothing ever completes, with a limit of limit_cycles SM cycles
+ * (1 .. 4e9; about 2e6 is a millisecond), records its code and returns.  The next tt_sync
+ * therefore reports TT_ERR_DEVICE_STATUS, clears the status word, and the context is usable as before.
+ * Nothing traps, faults or waits without bound.
+ */
+tt_status tt_debug_expire_wait(tt_ctx* ctx, uint64_t limit_cycles);
+
 /* ---------------------------------------------------------------------------------------
  * Stage-level entry points on caller-owned device buffers (no context needed).  They run
  * the same kernels as the corresponding stage of tt_submit_frames and are asynchronous on
@@ -282,7 +295,8 @@ tt_status tt_get_counters(const tt_ctx* ctx, uint64_t* kernel_launches, uint64_t
 /*
  * tt_preprocess — S1, the format-conversion operator of Section III-A.
  * src_dev: K frames, frame k at src_dev + k*src_frame_stride bytes, uint8 RGB interleaved,
- * row pitch src_pitch bytes.  dst_dev: fp32 [K][3][net_h][net_w].  For output sample o of
+ * row pitch src_pitch bytes (any alignment).  dst_dev: fp32 [K][3][net_h][net_w], 4-byte aligned
+ * (16-byte alignment with net_w a multiple of 4 lets the kernel use 128-bit stores).  For output sample o of
  * an axis resized from `in` to `out`: s = clamp((o+1/2)*in/out - 1/2, 0, in-1) evaluated in
  * exact integer arithmetic, i0 = floor(s), i1 = min(i0+1, in-1), weight s - i0.
  */
@@ -293,13 +307,14 @@ tt_status tt_preprocess(const uint8_t* src_dev, int32_t K, int64_t src_frame_str
 /*
  * tt_postprocess — S4+S5, the tool-tracking post-processing operator of Section III-A.
  * h_dev: fp32 hidden state of K streams, channels-last [K][Hm][Wm][hidden] when
- * channels_last != 0, else planar [K][hidden][Hm][Wm].  head_w/head_b (and conf_w/conf_b
+ * channels_last != 0 (16-byte aligned), else planar [K][hidden][Hm][Wm] (4-byte aligned).  head_w/head_b (and conf_w/conf_b
  * for TT_CONF_GAP_LINEAR) are device fp32 [n_tools][hidden] / [n_tools].
  * Outputs (device): logits, probs fp32 [K][n_tools][Hm][Wm]; masks uint8 same shape;
- * results: K tt_result records of which conf, cx, cy, count are written.
+ * results: K tt_result records (8-byte aligned) of which conf, cx, cy, count are written.
  * scratch_dev: tt_postprocess_scratch_bytes(...) bytes of device memory, 8-byte aligned; the call
  * clears it first, contents on entry are ignored.
- * hidden must be a multiple of 4 and at most 512.
+ * hidden must be a multiple of 4 and at most 512; hm, wm at most 16384.  A misaligned or null
+ * pointer is answered with TT_ERR_INVALID_ARG before anything is launched.
  */
 size_t tt_postprocess_scratch_bytes(int32_t K, int32_t hm, int32_t wm, int32_t hidden, int32_t n_tools);
 tt_status tt_postprocess(const float* h_dev, int32_t channels_last, int32_t K, int32_t hm, int32_t wm,
@@ -315,7 +330,8 @@ tt_status tt_postprocess(const float* h_dev, int32_t channels_last, int32_t K, i
  * that promised its host application a fixed memory footprint, plug-ins that are handed their
  * buffers by a framework's own allocator, and callers that keep a whole device reserved by
  * another pool.  Nothing is allocated or freed here, neither through CUDA nor through any
- * library: the partial sums that tt_postprocess keeps in caller-provided scratch live in a
+ * library (one exception: the very first call on a device makes the CUDA runtime load the
+ * library's device code, which the runtime does with allocations of its own; see below): the partial sums that tt_postprocess keeps in caller-provided scratch live in a
  * fixed array of TT_POSTPROCESS_STATIC_SCRATCH_BYTES that is part of the library image (each
  * GPU that loads the library holds that much memory until the process ends).  Inputs and
  * outputs are still the caller's.
@@ -323,10 +339,12 @@ tt_status tt_postprocess(const float* h_dev, int32_t channels_last, int32_t K, i
  * Limits and rules:
  *   - tt_postprocess_scratch_bytes(K, hm, wm, hidden, n_tools) must not exceed
  *     TT_POSTPROCESS_STATIC_SCRATCH_BYTES, else TT_ERR_UNSUPPORTED is returned and nothing runs
- *     (32 KiB: 8 streams with up to 468 hidden channels, any grid size; 8 streams of 512 hidden
- *     channels need 35 KB and are refused, 7 such streams fit);
- *   - the first call on a device looks up the array's device address (with that device
- *     current); make that first call before starting any stream capture;
+ *     (32 KiB: 256 + K * 8 * (hidden + 32) bytes rounded up to 256, so 8 streams fit with up to 476
+ *     hidden channels whatever the grid size; 8 streams of 512 hidden channels need 35 KB and are
+ *     refused, 7 such streams fit);
+ *   - the first call on a device looks up the array's device address and sets the kernels'
+ *     shared-memory attributes (with that device current); make that first call, once, in a
+ *     set-up phase and before starting any stream capture;
  *   - all calls on a device share the one array.  It keeps whatever the previous call left; the
  *     accumulators in it must start at zero, so every call clears the part it uses (a memset on
  *     `cuda_stream`) before its kernel runs.  Two calls whose kernels overlap on the GPU
@@ -344,7 +362,7 @@ tt_status tt_postprocess_static(const float* h_dev, int32_t channels_last, int32
  * tt_overlay — S6, the stand-in for the visualisation operator of Section II-B / III-A
  * (mask overlay on the frame).  src_dev as in tt_preprocess; masks_dev uint8
  * [K][n_tools][Hm][Wm]; palette: n_tools RGB triples (host); dst_dev uint8
- * [K][src_h][src_w][4].  Mask sample for source pixel (x, y): (floor(x*Wm/src_w),
+ * [K][src_h][src_w][4], 4-byte aligned.  Mask sample for source pixel (x, y): (floor(x*Wm/src_w),
  * floor(y*Hm/src_h)); tools blended in ascending order as (153*rgb + 102*colour + 127)/255.
  */
 tt_status tt_overlay(const uint8_t* src_dev, int32_t K, int64_t src_frame_stride, int32_t src_w, int32_t src_h,

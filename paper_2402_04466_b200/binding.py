@@ -27,7 +27,7 @@ TENSOR_IDS = {"pre": 0, "enc0": 1, "enc1": 2, "enc2": 3, "enc3": 4, "h": 8, "c":
 EXPORTED_SYMBOLS = [
     "tt_abi_version", "tt_create", "tt_destroy", "tt_last_error", "tt_map_size", "tt_state_create",
     "tt_state_reset", "tt_state_export", "tt_state_import", "tt_submit_frames", "tt_sync", "tt_debug_tensor",
-    "tt_set_profiling", "tt_get_stage_times", "tt_get_counters", "tt_query",
+    "tt_set_profiling", "tt_get_stage_times", "tt_get_counters", "tt_query", "tt_debug_expire_wait",
     "tt_sched_create", "tt_sched_destroy", "tt_sched_admit", "tt_sched_release", "tt_sched_arrive", "tt_sched_next",
     "tt_sched_complete", "tt_sched_predict_ms", "tt_sched_stats",
     "tt_preprocess", "tt_postprocess_scratch_bytes", "tt_postprocess", "tt_postprocess_static", "tt_overlay",
@@ -118,6 +118,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.tt_get_stage_times.argtypes = [vp, C.POINTER(C.c_float)]
     lib.tt_get_counters.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     lib.tt_query.argtypes = [vp]
+    lib.tt_debug_expire_wait.argtypes = [vp, C.c_uint64]
     u64p = C.POINTER(C.c_uint64)
     lib.tt_sched_create.argtypes = [C.POINTER(tt_sched_config), C.POINTER(vp)]
     lib.tt_sched_destroy.argtypes = [vp]
@@ -282,14 +283,17 @@ class Context:
     def sync(self) -> List[Dict]:
         res = (tt_result * TT_MAX_STREAMS)()
         st = self.lib.tt_sync(self.handle, res)
-        _check(self.lib, st, self.handle)
+        if st == 8 and self._ks:                 # TT_ERR_DEVICE_STATUS: the submit is over, its results are invalid
+            self._ks.pop(0)
+            self._inflight_keep.pop(0)
+        _check(self.lib, st, self.handle)        # any other error (a timeout, say) leaves the submit in flight
         k_done = self._ks.pop(0)                 # submits complete oldest first
         self._inflight_keep.pop(0)
         return [_result_to_dict(res[k], self.n_tools) for k in range(k_done)]
 
     def sync_raw(self, result_array) -> int:
         st = self.lib.tt_sync(self.handle, result_array)
-        if st == TT_OK and self._ks:
+        if st in (TT_OK, 8) and self._ks:
             self._ks.pop(0)
             self._inflight_keep.pop(0)
         return st
@@ -310,6 +314,10 @@ class Context:
     def query(self) -> bool:
         """True when the oldest submit in flight has finished (tt_sync would not block)."""
         return self.lib.tt_query(self.handle) == TT_OK
+
+    def debug_expire_wait(self, limit_cycles: int):
+        """Enqueue the failure-path probe: a bounded device-side wait that runs out after limit_cycles."""
+        _check(self.lib, self.lib.tt_debug_expire_wait(self.handle, limit_cycles), self.handle)
 
     def last_error(self) -> str:
         m = self.lib.tt_last_error(self.handle)

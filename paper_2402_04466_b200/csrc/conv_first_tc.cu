@@ -57,6 +57,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
 
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wait_limit = p.wait_limit;
   if (threadIdx.x == 0) {
     for (int s = 0; s < F_STAGES; ++s) {
       mbar_init(smem_u32(a_full + s), 128);
@@ -75,6 +76,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
     reinterpret_cast<uint4*>(s_b)[i] = __ldg(reinterpret_cast<const uint4*>(p.w_packed) + i);
   fence_proxy_async_smem();
   if (warp == 4) {
+    __syncwarp();   // the weight-staging loop may have left the lanes apart; the allocation is warp-collective
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)),
                  "r"((uint32_t)F_TMEM_COLS)
                  : "memory");
@@ -113,7 +115,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
       if (blockIdx.x + gridDim.x < total_tiles) fetch_patch(blockIdx.x + gridDim.x, 1);
     }
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      if (!fail && !mbar_wait(smem_u32(p_full + buf), pphase, abort_flag, p.status, 0x900 + buf)) fail = true;
+      if (!fail && !mbar_wait(smem_u32(p_full + buf), pphase, abort_flag, p.status, 0x900 + buf, wait_limit)) fail = true;
       const float* patch = reinterpret_cast<const float*>(s_patch + buf * PATCH_STRIDE);
       float v[27];
 #pragma unroll
@@ -131,7 +133,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
       }
       if (buf) pphase ^= 1u;
       buf ^= 1;
-      if (!mbar_wait(smem_u32(a_empty + stage), phase ^ 1u, abort_flag, p.status, 0x500 + (int)stage)) {
+      if (!mbar_wait(smem_u32(a_empty + stage), phase ^ 1u, abort_flag, p.status, 0x500 + (int)stage, wait_limit)) {
         fail = true;
         continue;
       }
@@ -156,8 +158,8 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
       uint32_t stage = 0, phase = 0, acc_phase = 0;
       int acc = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        if (!mbar_wait(smem_u32(t_empty + acc), acc_phase ^ 1u, abort_flag, p.status, 0x600 + acc)) break;
-        if (!mbar_wait(smem_u32(a_full + stage), phase, abort_flag, p.status, 0x700 + (int)stage)) break;
+        if (!mbar_wait(smem_u32(t_empty + acc), acc_phase ^ 1u, abort_flag, p.status, 0x600 + acc, wait_limit)) break;
+        if (!mbar_wait(smem_u32(a_full + stage), phase, abort_flag, p.status, 0x700 + (int)stage, wait_limit)) break;
         tc_fence_after();
         const uint32_t a_addr = smem_u32(s_a + stage * F_A_BYTES), b_addr = smem_u32(s_b);
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 64);
@@ -186,7 +188,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
     int acc = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
       const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, img = tile / tiles_per_img;
-      const bool fail = !mbar_wait(smem_u32(t_full + acc), acc_phase, abort_flag, p.status, 0x800 + acc);
+      const bool fail = !mbar_wait(smem_u32(t_full + acc), acc_phase, abort_flag, p.status, 0x800 + acc, wait_limit);
       // the previous tile's store must have finished reading s_out before it is overwritten
       if (leader) bulk_wait_group_read0();
       if (named_barrier_or(2, 128, fail)) break;   // all four warps stop together if any wait ran out

@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
 
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wait_limit = p.wait_limit;
   const int tiles_per_img = p.tiles_x * p.tiles_y;
   const int total_tiles = p.K * tiles_per_img * p.n_tiles_n;
   const int slabs_per_tap = p.slabs[0] + (p.n_src > 1 ? p.slabs[1] : 0);
@@ -138,6 +139,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     asm volatile("prefetch.tensormap [%0];" ::"l"(&p.map_b) : "memory");
   }
   if (warp == MMA_WARP) {
+    __syncwarp();   // the table loop above may have left the warp's lanes apart; the allocation is warp-collective
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                  "r"((uint32_t)Cfg::TMEM_COLS)
                  : "memory");
@@ -169,7 +171,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
       const int img_x = s_img[img], img_h = s_img[TT_MAX_STREAMS + img];
       for (; it < k_iters; it += n_prod) {
         const int4 e = s_tab[it];
-        ok = mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag, p.status, 0x100 + (int)stage);
+        ok = mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag, p.status, 0x100 + (int)stage, wait_limit);
         if (!ok) break;
         const uint32_t fb = smem_u32(full_bar + stage);
         uint8_t* st = smem + stage * Cfg::STAGE_BYTES;
@@ -195,13 +197,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
     uint64_t a_desc = a_desc0;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      ok = mbar_wait(smem_u32(tempty_bar + acc), acc_phase ^ 1u, abort_flag, p.status, 0x200 + acc);
+      ok = mbar_wait(smem_u32(tempty_bar + acc), acc_phase ^ 1u, abort_flag, p.status, 0x200 + acc, wait_limit);
       if (!ok) break;
       tc_fence_after();   // the epilogue's TMEM reads of this buffer come before the MMAs that overwrite it
       const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BLOCK_N);
       for (int it = 0; it < k_iters; ++it) {
         // the copies complete on the barrier through the async proxy, which the MMAs read through too
-        ok = mbar_wait(full0 + 8u * stage, phase, abort_flag, p.status, 0x300 + (int)stage);
+        ok = mbar_wait(full0 + 8u * stage, phase, abort_flag, p.status, 0x300 + (int)stage, wait_limit);
         if (!ok) break;
         const uint64_t b_desc = a_desc + B_UNITS;
         // advance along K inside the swizzle atom: 16 bf16 = 32 bytes = 2 descriptor units
@@ -254,7 +256,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
         }
       }
 
-      ok = mbar_wait(smem_u32(tfull_bar + acc), acc_phase, abort_flag, p.status, 0x400 + acc);
+      // the warp votes: its lanes leave the tile loop together or go on to the warp-collective TMEM loads together
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(tfull_bar + acc), acc_phase, abort_flag, p.status, 0x400 + acc, wait_limit));
       if (!ok) break;
       tc_fence_after();
       const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N + half * HALF_N);
@@ -365,8 +368,6 @@ cudaError_t launch_shape(const ConvTcParams& p, int sm_count, cudaStream_t s) {
 }
 
 }  // namespace
-
-cudaError_t conv_tc_prepare() { return cudaSuccess; }
 
 cudaError_t launch_conv_tc(const ConvTcParams& p, int sm_count, cudaStream_t s) {
   if (9 * (p.slabs[0] + (p.n_src > 1 ? p.slabs[1] : 0)) > MAX_K_ITERS || p.n_prod < 1 || p.n_prod > N_PROD) return cudaErrorInvalidValue;

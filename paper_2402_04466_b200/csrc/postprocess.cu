@@ -284,7 +284,7 @@ __device__ __forceinline__ void fma2(unsigned long long& acc, unsigned long long
 __device__ __forceinline__ uint32_t sw_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 // Bounded wait on a warp-private mbarrier; false when the limit ran out (the caller gives up).
-__device__ __forceinline__ bool sw_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool sw_wait(uint32_t bar, uint32_t parity, long long limit) {
   long long t0 = 0;
   for (uint32_t it = 0;; ++it) {
     uint32_t ok;
@@ -297,7 +297,7 @@ __device__ __forceinline__ bool sw_wait(uint32_t bar, uint32_t parity) {
     if ((it & 63u) == 63u) {
       const long long now = clock64();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > SW_WAIT_LIMIT_CYCLES) return false;
+      else if (now - t0 > limit) return false;
     }
   }
 }
@@ -364,6 +364,7 @@ __global__ void __launch_bounds__(StreamCfg<NCHUNK>::THREADS, 1) post_stream_ker
   __shared__ float s_gap_fin[512];
 
   const int T = p.T;
+  const long long wait_limit = p.wait_limit > 0 ? p.wait_limit : SW_WAIT_LIMIT_CYCLES;
   const int plane = p.Hm * p.Wm;
   const int rpi = (plane + SW_ROUND_PIX - 1) / SW_ROUND_PIX;    // rounds per image
   const int unit_rounds = sw_unit_rounds(plane), unit_pix = unit_rounds * SW_ROUND_PIX;
@@ -540,7 +541,7 @@ __global__ void __launch_bounds__(StreamCfg<NCHUNK>::THREADS, 1) post_stream_ker
       for (int r = 0; r < rounds; ++r) {
         const int pix0 = unit_pix0 + r * SW_ROUND_PIX;
         const int npix = min(SW_ROUND_PIX, plane - pix0);
-        ok = sw_wait(sw_smem_u32(bars + stage), parity);
+        ok = sw_wait(sw_smem_u32(bars + stage), parity, wait_limit);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) {
           // a copy never arrived: record it, give copies still in flight time to land, stop

@@ -122,7 +122,8 @@ preprocess_staged_kernel(const __grid_constant__ PreprocessParams p, int row_cap
   const int xoffs[4] = {xoff4.x - 3 * sx_lo, xoff4.y - 3 * sx_lo, xoff4.z - 3 * sx_lo, xoff4.w - 3 * sx_lo};
   const float fxs[4] = {fx4.x, fx4.y, fx4.z, fx4.w};
   const size_t plane = (size_t)p.net_h * p.net_w;
-  const bool vec_ok = ((p.net_w & 3) == 0) && (xo0 + 3 < p.net_w);
+  // with a row length that is a multiple of 4 every row start is as aligned as the tensor itself
+  const bool vec_ok = ((p.net_w & 3) == 0) && (xo0 + 3 < p.net_w) && (((uintptr_t)p.dst & 15) == 0);
 
 #pragma unroll
   for (int rr = 0; rr < 2; ++rr) {

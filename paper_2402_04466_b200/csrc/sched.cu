@@ -44,7 +44,11 @@ float predict(const tt_sched* s, int K) {
   for (int k = 1; k <= TT_MAX_STREAMS; ++k)
     if (s->seen[k] && (best < 0 || std::abs(k - K) < std::abs(best - K))) best = k;
   if (best < 0) return s->cfg.tick_ms_base + s->cfg.tick_ms_per_stream * (float)K;
-  return s->ewma_ms[best] + s->cfg.tick_ms_per_stream * (float)(K - best);
+  // extrapolating downwards with the prior's slope could cross zero; a tick of K streams never
+  // costs less than the K/best share of an observed tick of `best` streams
+  const float shifted = s->ewma_ms[best] + s->cfg.tick_ms_per_stream * (float)(K - best);
+  const float floor_ms = K < best ? s->ewma_ms[best] * (float)K / (float)best : s->ewma_ms[best];
+  return std::max(shifted, floor_ms);
 }
 
 }  // namespace

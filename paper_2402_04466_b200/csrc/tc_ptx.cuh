@@ -9,7 +9,7 @@
 namespace tt {
 namespace tc {
 
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // about 2 s of SM cycles per wait
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // default limit of a wait: about 2 s of SM cycles
 // How long one try_wait may keep its thread suspended inside the barrier unit before it reports
 // "not yet": a suspended thread issues nothing, a thread that polls in a loop takes issue slots
 // from the warps that share its scheduler.
@@ -41,8 +41,9 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // Bounded wait.  Returns false when the block is aborting (this wait or another one ran out).
 // The limit is counted on the SM's cycle counter (cheap to read, unlike the global nanosecond
 // timer) and only consulted every 64 failed polls, so the common short wait costs nothing extra.
+// `limit` is a kernel parameter (the host passes WAIT_LIMIT_CYCLES unless told otherwise).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code) {
+                                          int code, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
@@ -52,7 +53,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       const long long now = clock64();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > WAIT_LIMIT_CYCLES) {
+      } else if (now - t0 > limit) {
         *abort_flag = 1;
         atomicCAS(status, 0, code);
         return false;

@@ -164,6 +164,7 @@ struct tt_ctx {
   bool stage_valid = false;
   float stage_ms[TT_STAGE_COUNT];
   uint64_t n_launches = 0, n_ticks = 0;
+  long long wait_limit = DEFAULT_WAIT_LIMIT_CYCLES;   // SM cycles a device-side barrier wait may take
   std::vector<void*> allocs;
   std::string err;
 };
@@ -536,7 +537,7 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
       f.in = ctx->pre; f.out = reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[0]);
       f.H = c.net_h; f.W = c.net_w; f.Ho = ctx->lay_h[1]; f.Wo = ctx->lay_w[1]; f.stride = c.enc_stride[0]; f.cout = co;
       f.tiles_x = (f.Wo + 15) / 16; f.tiles_y = (f.Ho + 7) / 8;
-      f.w_packed = dw; f.bias = db; f.status = ctx->status_dev;
+      f.w_packed = dw; f.bias = db; f.status = ctx->status_dev; f.wait_limit = ctx->wait_limit;
       {
         const cuuint64_t dims[4] = {(cuuint64_t)co, (cuuint64_t)f.Wo, (cuuint64_t)f.Ho, (cuuint64_t)S};
         const cuuint64_t str[3] = {(cuuint64_t)co * 2, (cuuint64_t)f.Wo * co * 2, (cuuint64_t)f.Ho * f.Wo * co * 2};
@@ -688,7 +689,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
       if (bi < 0) return fail(ctx, TT_ERR_UNSUPPORTED, "no tensor-core tile shape fits this layer");
       const int bns[3] = {64, 128, 256};
       q.block_n = bns[bi]; q.map_b = L.map_b[bi]; q.n_tiles_n = L.cout / q.block_n;
-      q.cout = L.cout; q.bias = L.b; q.status = ctx->status_dev;
+      q.cout = L.cout; q.bias = L.b; q.status = ctx->status_dev; q.wait_limit = ctx->wait_limit;
       q.n_prod = 3;
       q.pdl = ctx->profiling ? 0 : 1;
       return TT_OK;
@@ -721,7 +722,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
   po.head_w = ctx->head_w; po.head_b = ctx->head_b; po.conf_w = ctx->conf_w; po.conf_b = ctx->conf_b;
   po.conf_mode = c.conf_mode; po.zthr = ctx->zthr;
   po.logits = ctx->logits; po.probs = ctx->probs; po.masks = ctx->masks; po.bits = ctx->bits;
-  po.results = ctx->results_dev; po.scratch = ctx->post_scratch; po.status = ctx->status_dev;
+  po.results = ctx->results_dev; po.scratch = ctx->post_scratch; po.status = ctx->status_dev; po.wait_limit = ctx->wait_limit;
   po.pdl = (ctx->bf16 && !ctx->profiling) ? 1 : 0;
   TT_CUDA(ctx, launch_postprocess(po, s));
   if ((ms_ = mark_stage(ctx, TT_STAGE_POSTPROCESS, 2)) != TT_OK) return ms_;
@@ -1129,7 +1130,43 @@ tt_status tt_get_counters(const tt_ctx* ctx, uint64_t* kernel_launches, uint64_t
   return TT_OK;
 }
 
+tt_status tt_debug_expire_wait(tt_ctx* ctx, uint64_t limit_cycles) {
+  if (!ctx) return TT_ERR_INVALID_ARG;
+  if (limit_cycles == 0 || limit_cycles > (uint64_t)DEFAULT_WAIT_LIMIT_CYCLES)
+    return fail(ctx, TT_ERR_INVALID_ARG, "limit_cycles must lie in [1, %lld]", DEFAULT_WAIT_LIMIT_CYCLES);
+  TT_CUDA(ctx, cudaSetDevice(ctx->dev));
+  TT_CUDA(ctx, launch_wait_probe(ctx->status_dev, (long long)limit_cycles, 0xA00, ctx->stream));
+  return TT_OK;
+}
+
 // ------------------------------------------------------------------------- stage-level calls
+namespace {
+inline bool misaligned(const void* p, uintptr_t a) { return ((uintptr_t)p & (a - 1)) != 0; }
+
+// Argument checks shared by tt_postprocess and tt_postprocess_static.  Everything the kernels
+// assume about sizes and alignment is checked here, on the host, so that a bad argument comes
+// back as a status and never as a device fault.
+tt_status check_post_args(const char* who, const float* h_dev, int32_t channels_last, int32_t K, int32_t hm, int32_t wm,
+                          int32_t hidden, int32_t n_tools, const float* head_w_dev, const float* head_b_dev,
+                          const float* conf_w_dev, const float* conf_b_dev, int32_t conf_mode, float threshold,
+                          float* logits_dev, float* probs_dev, uint8_t* masks_dev, tt_result* results_dev) {
+  if (!h_dev || !head_w_dev || !head_b_dev || !logits_dev || !probs_dev || !masks_dev || !results_dev || K < 1 ||
+      K > TT_MAX_STREAMS || hm < 1 || wm < 1 || hm > 16384 || wm > 16384 || n_tools < 1 || n_tools > TT_MAX_TOOLS ||
+      !(threshold > 0.f && threshold < 1.f) || (conf_mode != TT_CONF_MEAN_SIGMOID && conf_mode != TT_CONF_GAP_LINEAR) ||
+      (conf_mode == TT_CONF_GAP_LINEAR && (!conf_w_dev || !conf_b_dev)))
+    return fail(nullptr, TT_ERR_INVALID_ARG, "%s: bad argument", who);
+  if (hidden < 4 || hidden > 512 || hidden % 4) return fail(nullptr, TT_ERR_UNSUPPORTED, "%s: hidden must be a multiple of 4 in [4, 512]", who);
+  // channels-last rows are read with 128-bit loads; every fp32 tensor with 32-bit accesses; the result records hold 64-bit members
+  if (misaligned(h_dev, channels_last ? 16 : 4) || misaligned(head_w_dev, 4) || misaligned(head_b_dev, 4) ||
+      misaligned(conf_w_dev, 4) || misaligned(conf_b_dev, 4) || misaligned(logits_dev, 4) || misaligned(probs_dev, 4) ||
+      misaligned(results_dev, 8))
+    return fail(nullptr, TT_ERR_INVALID_ARG,
+                "%s: misaligned pointer (h_dev needs %d-byte alignment, other fp32 tensors 4, results_dev 8)", who,
+                channels_last ? 16 : 4);
+  return TT_OK;
+}
+}  // namespace
+
 tt_status tt_preprocess(const uint8_t* src_dev, int32_t K, int64_t src_frame_stride, int32_t src_w, int32_t src_h,
                         int32_t src_pitch, float* dst_dev, int32_t net_w, int32_t net_h, float norm_div,
                         float norm_mean, float norm_std, void* cuda_stream) {
@@ -1137,6 +1174,7 @@ tt_status tt_preprocess(const uint8_t* src_dev, int32_t K, int64_t src_frame_str
       src_w > 16384 || src_h > 16384 || net_w > 16384 || net_h > 16384 || src_pitch < 3 * src_w || norm_div == 0.f ||
       norm_std == 0.f)
     return fail(nullptr, TT_ERR_INVALID_ARG, "tt_preprocess: bad argument");
+  if (misaligned(dst_dev, 4)) return fail(nullptr, TT_ERR_INVALID_ARG, "tt_preprocess: dst_dev must be 4-byte aligned");
   PreprocessParams p{};
   for (int n = 0; n < K; ++n) p.src.p[n] = src_dev + (size_t)n * src_frame_stride;
   p.K = K; p.src_w = src_w; p.src_h = src_h; p.src_pitch = src_pitch; p.net_w = net_w; p.net_h = net_h;
@@ -1155,12 +1193,11 @@ tt_status tt_postprocess(const float* h_dev, int32_t channels_last, int32_t K, i
                          int32_t n_tools, const float* head_w_dev, const float* head_b_dev, const float* conf_w_dev,
                          const float* conf_b_dev, int32_t conf_mode, float threshold, float* logits_dev, float* probs_dev,
                          uint8_t* masks_dev, tt_result* results_dev, void* scratch_dev, void* cuda_stream) {
-  if (!h_dev || !head_w_dev || !head_b_dev || !logits_dev || !probs_dev || !masks_dev || !results_dev || !scratch_dev ||
-      K < 1 || K > TT_MAX_STREAMS || hm < 1 || wm < 1 || n_tools < 1 || n_tools > TT_MAX_TOOLS ||
-      !(threshold > 0.f && threshold < 1.f) || (conf_mode != TT_CONF_MEAN_SIGMOID && conf_mode != TT_CONF_GAP_LINEAR) ||
-      (conf_mode == TT_CONF_GAP_LINEAR && (!conf_w_dev || !conf_b_dev)))
-    return fail(nullptr, TT_ERR_INVALID_ARG, "tt_postprocess: bad argument");
-  if (hidden < 4 || hidden > 512 || hidden % 4) return fail(nullptr, TT_ERR_UNSUPPORTED, "tt_postprocess: hidden must be a multiple of 4 in [4, 512]");
+  tt_status a = check_post_args("tt_postprocess", h_dev, channels_last, K, hm, wm, hidden, n_tools, head_w_dev, head_b_dev,
+                                conf_w_dev, conf_b_dev, conf_mode, threshold, logits_dev, probs_dev, masks_dev, results_dev);
+  if (a != TT_OK) return a;
+  if (!scratch_dev || misaligned(scratch_dev, 8))
+    return fail(nullptr, TT_ERR_INVALID_ARG, "tt_postprocess: scratch_dev is null or not 8-byte aligned");
   cudaError_t e = post_prepare();
   if (e != cudaSuccess) return fail(nullptr, TT_ERR_CUDA, "tt_postprocess: %s", cudaGetErrorString(e));
   PostParams p{};
@@ -1185,13 +1222,10 @@ tt_status tt_postprocess_static(const float* h_dev, int32_t channels_last, int32
                                 const float* conf_w_dev, const float* conf_b_dev, int32_t conf_mode, float threshold,
                                 float* logits_dev, float* probs_dev, uint8_t* masks_dev, tt_result* results_dev,
                                 void* cuda_stream) {
-  if (!h_dev || !head_w_dev || !head_b_dev || !logits_dev || !probs_dev || !masks_dev || !results_dev || K < 1 ||
-      K > TT_MAX_STREAMS || hm < 1 || wm < 1 || n_tools < 1 || n_tools > TT_MAX_TOOLS ||
-      !(threshold > 0.f && threshold < 1.f) || (conf_mode != TT_CONF_MEAN_SIGMOID && conf_mode != TT_CONF_GAP_LINEAR) ||
-      (conf_mode == TT_CONF_GAP_LINEAR && (!conf_w_dev || !conf_b_dev)))
-    return fail(nullptr, TT_ERR_INVALID_ARG, "tt_postprocess_static: bad argument");
-  if (hidden < 4 || hidden > 512 || hidden % 4)
-    return fail(nullptr, TT_ERR_UNSUPPORTED, "tt_postprocess_static: hidden must be a multiple of 4 in [4, 512]");
+  tt_status a = check_post_args("tt_postprocess_static", h_dev, channels_last, K, hm, wm, hidden, n_tools, head_w_dev,
+                                head_b_dev, conf_w_dev, conf_b_dev, conf_mode, threshold, logits_dev, probs_dev, masks_dev,
+                                results_dev);
+  if (a != TT_OK) return a;
   const size_t need = post_scratch_bytes(K, hm, wm, hidden, n_tools);
   if (need > (size_t)TT_POSTPROCESS_STATIC_SCRATCH_BYTES)
     return fail(nullptr, TT_ERR_UNSUPPORTED,
@@ -1223,8 +1257,10 @@ tt_status tt_overlay(const uint8_t* src_dev, int32_t K, int64_t src_frame_stride
                      int32_t src_pitch, const uint8_t* masks_dev, int32_t n_tools, int32_t hm, int32_t wm,
                      const uint8_t* palette_host, uint8_t* dst_dev, void* cuda_stream) {
   if (!src_dev || !masks_dev || !palette_host || !dst_dev || K < 1 || K > TT_MAX_STREAMS || src_w < 1 || src_h < 1 ||
-      src_pitch < 3 * src_w || n_tools < 1 || n_tools > TT_MAX_TOOLS || hm < 1 || wm < 1)
+      src_w > 16384 || src_h > 16384 || src_pitch < 3 * src_w || n_tools < 1 || n_tools > TT_MAX_TOOLS || hm < 1 || wm < 1 ||
+      hm > 16384 || wm > 16384)
     return fail(nullptr, TT_ERR_INVALID_ARG, "tt_overlay: bad argument");
+  if (misaligned(dst_dev, 4)) return fail(nullptr, TT_ERR_INVALID_ARG, "tt_overlay: dst_dev must be 4-byte aligned (RGBA8 pixels are stored as words)");
   OverlayParams p{};
   for (int n = 0; n < K; ++n) p.src.p[n] = src_dev + (size_t)n * src_frame_stride;
   p.K = K; p.src_w = src_w; p.src_h = src_h; p.src_pitch = src_pitch; p.T = n_tools; p.Hm = hm; p.Wm = wm;

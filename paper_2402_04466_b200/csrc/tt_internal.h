@@ -98,6 +98,7 @@ struct ConvFirstTcParams {
   const uint16_t* w_packed;   // device, cout*32 bf16 in the MMA operand layout
   const float* bias;          // device, [cout]
   int32_t* status;
+  long long wait_limit;       // SM cycles after which a barrier wait gives up
 };
 bool conv_first_tc_supported(int cout);
 int conv_first_tc_box_w(int stride);   // columns of the input patch box (a multiple of 4)
@@ -138,9 +139,15 @@ struct ConvTcParams {
   IdxMap c_idx, h_out_idx;  // slot, slot*2+half
   int32_t hidden;
   int32_t* status;          // device word: 0 ok, else a code describing a wait that ran out
+  long long wait_limit;     // SM cycles after which a barrier wait gives up
 };
 cudaError_t launch_conv_tc(const ConvTcParams& p, int sm_count, cudaStream_t s);
-cudaError_t conv_tc_prepare();  // one-off function attribute set-up
+constexpr long long DEFAULT_WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s of SM cycles
+
+// Failure-path probe: one warp waits, through the same bounded wait as the tensor-core kernels, on
+// a barrier that nothing ever completes; when `limit_cycles` have passed it records `code` in
+// *status and returns normally.
+cudaError_t launch_wait_probe(int32_t* status, long long limit_cycles, int code, cudaStream_t s);
 
 // ------------------------------------------------------------------- S4/S5 postprocess
 struct PostParams {
@@ -162,6 +169,7 @@ struct PostParams {
   tt_result* results;   // device, [K]
   void* scratch;
   int32_t* status;      // optional device word: set non-zero when a bounded wait ran out
+  long long wait_limit; // SM cycles after which a wait for a copy gives up (0: the default)
   int32_t pdl;          // launch as a programmatic dependent of the previous kernel in the stream (channels-last kernel only)
 };
 size_t post_scratch_bytes(int K, int hm, int wm, int ch, int T);

@@ -26,11 +26,19 @@ def _frames(wl, K, n):
     return [tt_synth.make_frames(wl.frame_kind, wl.stream_seed(s), n, wl.src_w, wl.src_h) for s in range(K)]
 
 
-def _compare_frame(ctx, st, res, ref, tol, band, check_tensors=True, tag="", tol_mid=None):
+# Every frame compared with the oracle leaves a record here; conftest prints the maxima at the end of the
+# run (how many mask pixels differ and how far from the threshold the oracle's logit is there), which is
+# what the width of the bf16 mask band is derived from.
+FLIP_LOG = []
+
+
+def _compare_frame(ctx, st, res, ref, tol, band, check_tensors=True, tag="", tol_mid=None, max_band_frac=None, log=True):
     """One stream, one frame: every observable of the CUDA path against the oracle's FrameOutput.
 
     tol bounds the path's float outputs (probabilities, confidences); tol_mid (default: tol)
-    bounds the intermediate tensors read through the debug taps.
+    bounds the intermediate tensors read through the debug taps.  Masks must agree wherever the
+    oracle's logit is at least `band` away from the threshold; max_band_frac bounds the share of
+    pixels inside that band (a band that swallows the mask would make the check vacuous).
     """
     stats = {}
     tol_mid = tol if tol_mid is None else tol_mid
@@ -46,12 +54,24 @@ def _compare_frame(ctx, st, res, ref, tol, band, check_tensors=True, tag="", tol
     gm = ctx.fetch_masks(res)
     zthr = float(np.log(ctx.cfg.threshold / (1.0 - ctx.cfg.threshold)))
     stats["band_frac"] = check_masks(gm, ref.mask, ref.z, zthr, band, tag + " mask")
+    if max_band_frac is not None:
+        assert stats["band_frac"] < max_band_frac, f"{tag}: {stats['band_frac']:.3%} of the pixels lie inside the mask band"
     check_reductions_from_own_mask(res, gm)
-    flips = int((gm != ref.mask).sum())
+    flipped = gm != ref.mask
+    flips = int(flipped.sum())
     stats["flips"] = flips
+    margin = float(np.abs(ref.z.astype(np.float64) - zthr)[flipped].max()) if flips else 0.0
+    z_rms = float(np.sqrt(np.mean(ref.z.astype(np.float64) ** 2)))
+    stats["flip_margin"] = margin
+    stats["flip_margin_rel"] = margin / max(z_rms, 1e-30)
+    if log:
+        FLIP_LOG.append({"tag": tag, "flips": flips, "pixels": int(gm.size), "margin": margin, "margin_rel": margin / max(z_rms, 1e-30),
+                         "band": band, "band_frac": stats["band_frac"], "tol": tol})
     for t in range(gm.shape[0]):
         n_ref = int(ref.count[t])
-        if n_ref > 0 and res["count"][t] > 0 and flips * 100 < n_ref:
+        flips_t = int(flipped[t].sum())
+        # threshold-sensitive pixels move the centroid; it is compared while they are under 1 % of the tool's mask
+        if n_ref > 0 and res["count"][t] > 0 and flips_t * 100 < n_ref:
             assert abs(res["cx"][t] - ref.cx[t]) <= 0.5 and abs(res["cy"][t] - ref.cy[t]) <= 0.5, (tag, t)
     return stats
 
@@ -113,6 +133,10 @@ def test_fp32_path_stride2_multistream_pinned_host_frames(cuda_device):
 # elements of c, h and the encoder maps by up to 3e-2 of the tensor rms (the oracle shows
 # this on its own, see test_oracle_bf16_rounding_spread).
 TOL_OUT, TOL_MID_PLAIN, TOL_MIRROR, TOL_MIRROR_RMS = 2e-2, 5e-2, 2e-2, 3e-3
+# Mask band of the bf16 path: masks must equal the oracle's wherever the oracle's logit is farther than
+# max(1e-3, BAND_REL * rms(z)) from the threshold, and on gain-corrected weights (logits of O(1) spread) less
+# than MAX_BAND_FRAC of the pixels may lie inside that band.
+BAND_REL, MAX_BAND_FRAC = 2e-2, 0.05
 
 
 def _run_bf16(cuda_device, wl, K, n_frames, tol_plain=TOL_OUT, tol_mirror=TOL_MIRROR, overlay=False):
@@ -129,14 +153,15 @@ def _run_bf16(cuda_device, wl, K, n_frames, tol_plain=TOL_OUT, tol_mirror=TOL_MI
             ref = plain[k].step(frames[k][t], want_overlay=False)
             # the stated bf16 tolerance against the fp32-activation oracle; masks may differ only
             # where the logit lies within the same tolerance of the threshold
-            band = max(1e-3, tol_plain * float(np.sqrt(np.mean(ref.z.astype(np.float64) ** 2))))
+            band = max(1e-3, BAND_REL * float(np.sqrt(np.mean(ref.z.astype(np.float64) ** 2))))
             s = _compare_frame(ctx, states[k], res[k], ref, tol_plain, band, tag=f"{wl.name} plain k={k} t={t}",
-                               tol_mid=TOL_MID_PLAIN)
+                               tol_mid=TOL_MID_PLAIN, max_band_frac=MAX_BAND_FRAC if wl.gain_corrected else None)
             refm = mirror[k].step(frames[k][t], want_overlay=False)
             # both sides rounding the same activations to bf16: only accumulation order and the
-            # fast transcendentals differ
+            # fast transcendentals differ (a diagnostic: this oracle variant rounds where the kernels
+            # round, so no parity claim rests on it)
             bandm = max(1e-3, tol_mirror * float(np.sqrt(np.mean(refm.z.astype(np.float64) ** 2))))
-            sm = _compare_frame(ctx, states[k], res[k], refm, tol_mirror, bandm, tag=f"{wl.name} mirror k={k} t={t}")
+            sm = _compare_frame(ctx, states[k], res[k], refm, tol_mirror, bandm, tag=f"{wl.name} mirror k={k} t={t}", log=False)
             for name, want in (("h", refm.h), ("c", refm.c), ("logits", refm.z)):
                 e = rms_err(ctx.debug_tensor(states[k], name), want)
                 assert e <= TOL_MIRROR_RMS, f"{wl.name} mirror k={k} t={t} {name}: rms error {e:.3e}"
@@ -231,9 +256,9 @@ def test_cfg2_five_streams_match_single_stream_runs(cuda_device):
         res = ctx.sync()
         refs = [oras[k].step(frames[k][t], want_overlay=False) for k in range(K)]
         for k in range(K):
-            band = max(1e-3, 2e-2 * float(np.sqrt(np.mean(refs[k].z.astype(np.float64) ** 2))))
+            band = max(1e-3, BAND_REL * float(np.sqrt(np.mean(refs[k].z.astype(np.float64) ** 2))))
             _compare_frame(ctx, states[k], res[k], refs[k], TOL_OUT, band, check_tensors=(t == n - 1),
-                           tag=f"cfg2 k={k} t={t}", tol_mid=TOL_MID_PLAIN)
+                           tag=f"cfg2 k={k} t={t}", tol_mid=TOL_MID_PLAIN, max_band_frac=MAX_BAND_FRAC)
         batched.append([(ctx.fetch_probs(r), r["conf"].copy(), r["count"].copy()) for r in res])
     h_b = [ctx.state_export(s) for s in states]
     ctx.destroy()
@@ -268,8 +293,8 @@ def test_teacher_forced_late_frame_and_state_roundtrip(cuda_device):
     ctx.submit_frames([torch.from_numpy(frames[6]).to(cuda_device)], [st], frame_index=306)
     (res,) = ctx.sync()
     ref = ora.step(frames[6], want_overlay=False)
-    band = max(1e-3, 2e-2 * float(np.sqrt(np.mean(ref.z.astype(np.float64) ** 2))))
-    _compare_frame(ctx, st, res, ref, TOL_OUT, band, tag="teacher-forced", tol_mid=TOL_MID_PLAIN)
+    band = max(1e-3, BAND_REL * float(np.sqrt(np.mean(ref.z.astype(np.float64) ** 2))))
+    _compare_frame(ctx, st, res, ref, TOL_OUT, band, tag="teacher-forced", tol_mid=TOL_MID_PLAIN, max_band_frac=MAX_BAND_FRAC)
     ctx.state_reset(st)
     h0, c0 = ctx.state_export(st)
     assert not h0.any() and not c0.any()
@@ -459,6 +484,76 @@ def test_boundary_error_paths(cuda_device):
     with pytest.raises(binding.TTError) as e:
         binding.Context(binding.make_config(bad), tt_synth.make_weights(bad))
     assert e.value.status == 2
+
+
+def test_host_side_sync_timeout_leaves_the_submit_in_flight(cuda_device):
+    """Failure detection on the host: with sync_timeout_ns = 1 us the first tt_sync of a scale-sweep-sized tick
+    gives up with TT_ERR_TIMEOUT (nothing is lost, the submit stays in flight); repeating the call until it
+    succeeds returns exactly what a context without a timeout returns."""
+    wl = tt_synth.workload("cfg4-gain")
+    fr = torch.from_numpy(tt_synth.make_frame(wl.frame_kind, wl.stream_seed(0), 0, wl.src_w, wl.src_h)).to(cuda_device)
+    ctx_ref, (st_ref,), _ = _make(wl)
+    ctx_ref.submit_frames([fr], [st_ref])
+    (want,) = ctx_ref.sync()
+    want_p = ctx_ref.fetch_probs(want)
+    ctx, (st,), _ = _make(wl, timeout_ns=1000)
+    ctx.submit_frames([fr], [st])                                 # first tick of a context: plain launches, > 100 us of GPU work
+    with pytest.raises(binding.TTError) as e:
+        ctx.sync()
+    assert e.value.status == 7 and "timed out" in str(e.value)
+    with pytest.raises(binding.TTError) as e:
+        ctx.state_export(st)                                      # the submit is still in flight
+    assert e.value.status == 6
+    res, tries = None, 0
+    while res is None:
+        try:
+            (res,) = ctx.sync()
+        except binding.TTError as err:
+            assert err.status == 7
+            tries += 1
+            assert tries < 10_000_000
+    assert np.array_equal(ctx.fetch_probs(res), want_p)
+    assert np.array_equal(res["conf"], want["conf"]) and np.array_equal(res["count"], want["count"])
+    with pytest.raises(binding.TTError) as e:
+        ctx.sync()
+    assert e.value.status == 6                                    # nothing left in flight
+    ctx.destroy()
+    ctx_ref.destroy()
+
+
+def test_device_side_wait_that_runs_out_is_reported_and_the_context_recovers(cuda_device):
+    """Failure detection on the device, in the form that harms nothing: a probe warp waits through the kernels'
+    own bounded barrier wait on a barrier that nothing completes, with a limit of about a millisecond.  It gives
+    up, records its code and returns; the tick behind it is answered with TT_ERR_DEVICE_STATUS; the tick after
+    that runs normally and matches the oracle."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="waitprobe", src_w=214, src_h=120, net_w=160, net_h=120, hidden=64)
+    ctx, (st,), w = _make(wl)
+    ora = oracle.OraclePipeline(wl, w)
+    frames = _frames(wl, 1, 4)[0]
+
+    def tick(t):
+        ctx.submit_frames([torch.from_numpy(frames[t]).to(cuda_device)], [st], frame_index=t)
+        return ctx.sync()[0]
+
+    def check(res, ref, t):
+        band = max(1e-3, BAND_REL * float(np.sqrt(np.mean(ref.z.astype(np.float64) ** 2))))
+        _compare_frame(ctx, st, res, ref, TOL_OUT, band, tag=f"waitprobe t={t}", tol_mid=TOL_MID_PLAIN)
+
+    check(tick(0), ora.step(frames[0], want_overlay=False), 0)
+    ctx.debug_expire_wait(2_000_000)                              # about 1 ms of SM cycles
+    with pytest.raises(binding.TTError) as e:
+        tick(1)
+    assert e.value.status == 8 and "0xa00" in str(e.value).lower()
+    ora.step(frames[1], want_overlay=False)                       # the tick itself ran; only its report was poisoned
+    with pytest.raises(binding.TTError) as e:
+        ctx.sync()
+    assert e.value.status == 6                                    # that submit is over
+    check(tick(2), ora.step(frames[2], want_overlay=False), 2)   # status word cleared: the context works as before
+    check(tick(3), ora.step(frames[3], want_overlay=False), 3)
+    with pytest.raises(binding.TTError) as e:
+        ctx.debug_expire_wait(0)
+    assert e.value.status == 1
+    ctx.destroy()
 
 
 def test_staggered_arrivals_through_the_planner_match_per_stream_runs(cuda_device):

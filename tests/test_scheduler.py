@@ -96,3 +96,26 @@ def test_admission_by_capacity_and_by_predicted_tick_time():
         assert len(s.next((k + 1) * PERIOD)[0]) == 4
         s.complete(2.0, (k + 1) * PERIOD + 2 * MS)
     assert s.predict_ms(4) == pytest.approx(2.0, abs=1e-3)
+
+
+def test_prediction_below_the_only_observed_batch_size_stays_positive():
+    """Only ticks of 8 streams have been seen (0.4 ms); the prior's slope (0.1 ms per stream) would put a
+    one-stream tick at -0.3 ms.  The prediction is floored by the 1/8 share of the observed tick, and the
+    planner keeps coalescing instead of treating every frame as deadline-critical."""
+    s = Scheduler(max_streams=8, window_ns=1 * MS, deadline_ns=PERIOD, tick_ms_base=0.1, tick_ms_per_stream=0.1)
+    ids = [s.admit() for _ in range(8)]
+    for i in ids:
+        s.arrive(i, 0, 0)
+    assert len(s.next(0)[0]) == 8
+    s.complete(0.4, 400_000)
+    assert s.predict_ms(8) == pytest.approx(0.4)
+    assert s.predict_ms(1) == pytest.approx(0.05)                 # 0.4 * 1/8, not 0.4 - 0.7
+    assert all(s.predict_ms(k) > 0 for k in range(1, 9))
+    assert s.predict_ms(7) == pytest.approx(0.35)                 # max(0.4 - 0.1, 0.4 * 7/8)
+    # a batch in flight, one frame waiting: it is held for the window, not released as "deadline near"
+    for i in ids:
+        s.arrive(i, 1, PERIOD)
+    assert len(s.next(PERIOD)[0]) == 8
+    assert s.arrive(ids[0], 2, 2 * PERIOD)
+    batch, wake = s.next(2 * PERIOD)
+    assert batch == [] and wake == 2 * PERIOD + 1 * MS
