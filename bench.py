@@ -31,6 +31,8 @@ if ROOT not in sys.path:
 METRIC = "frames/s over K streams"
 UNIT = "frames/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# plain fp32 arithmetic: 148 multiprocessors x 128 FMA lanes x 2 flops at the 1965 MHz maximum clock (derived, not measured)
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 FRAME_PERIOD_NS = 16_666_667
 
 
@@ -156,8 +158,19 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------ CPU oracle
-def time_oracle(wl, budget_s=12.0, max_frames=8):
-    """The oracle as it stands, on a bounded sample: whole stream-frames of this workload."""
+def cpu_model():
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def time_oracle(wl, budget_s=12.0, max_frames=8, single_thread_frames=1):
+    """The oracle as it stands, on a bounded sample: whole stream-frames of this workload, first on all
+    host threads the oracle uses, then on one thread."""
     import oracle
     import tt_synth
     w = tt_synth.make_weights(wl)
@@ -169,9 +182,25 @@ def time_oracle(wl, budget_s=12.0, max_frames=8):
         pipe.step(fr)
         t_total += time.perf_counter() - t0
         n += 1
-    return {"value": n / t_total, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"{n} stream-frames of {wl.name} (one stream, consecutive frames) in {t_total:.1f} s; "
-                      "per-frame cost is independent of K, so K streams cost K times as much"}
+    threads = oracle.num_threads()
+    out = {"value": n / t_total, "unit": UNIT, "cores": threads, "kind": "oracle", "cpu_model": cpu_model(),
+           "host_cpus": os.cpu_count(),
+           "sample": f"{n} stream-frames of {wl.name} (one stream, consecutive frames) in {t_total:.1f} s; "
+                     "per-frame cost is independent of K, so K streams cost K times as much"}
+    if single_thread_frames > 0:
+        oracle.set_threads(1)
+        try:
+            t1 = 0.0
+            for i in range(single_thread_frames):
+                fr = tt_synth.make_frame(wl.frame_kind, wl.stream_seed(0), n + i, wl.src_w, wl.src_h)
+                t0 = time.perf_counter()
+                pipe.step(fr)
+                t1 += time.perf_counter() - t0
+        finally:
+            oracle.set_threads(threads)
+        out["single_thread"] = {"value": single_thread_frames / t1, "unit": UNIT, "cores": 1,
+                                "sample": f"{single_thread_frames} stream-frame(s) of {wl.name} in {t1:.1f} s"}
+    return out
 
 
 def run_reference(args):
@@ -204,8 +233,10 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 0, "steps": len(times),
             "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": describe(wl, K), "note": "one stream-frame per step; oracle cost scales linearly in K"},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "config": {"workload": describe(wl, K)},
+            "note": "one stream-frame per step; oracle cost scales linearly in K",
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample,
+                             "cpu_model": cpu_model()},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
     return 0
@@ -220,10 +251,12 @@ def paced_run(ctx, states, host_ring, K, R, n_frames):
 
     from paper_2402_04466_b200 import binding
     from paper_2402_04466_b200.stats import latency_summary, trim_warmup
+    pinned_cpu = None
     try:
-        os.sched_setaffinity(0, {sorted(os.sched_getaffinity(0))[-1]})
+        pinned_cpu = sorted(os.sched_getaffinity(0))[-1]
+        os.sched_setaffinity(0, {pinned_cpu})
     except Exception:
-        pass
+        pinned_cpu = None
     fr = (binding.tt_frame * K)()
     sts = (C.c_void_p * K)(*[s.value for s in states])
     res = (binding.tt_result * binding.TT_MAX_STREAMS)()
@@ -248,7 +281,7 @@ def paced_run(ctx, states, host_ring, K, R, n_frames):
         misses += int(done - arrival > FRAME_PERIOD_NS)
     latency = latency_summary(trim_warmup(lat_ms))
     latency.update({"streams": K, "frames_per_stream": n_frames, "frame_period_ms": FRAME_PERIOD_NS / 1e6,
-                    "deadline_misses": misses, "gpu_ms_mean": float(np.mean(trim_warmup(gpu_ms))),
+                    "deadline_misses": misses, "gpu_ms_mean": float(np.mean(trim_warmup(gpu_ms))), "pacing_thread_cpu": pinned_cpu,
                     "definition": "scheduled arrival of the K frames -> tt_sync returned (pinned host frames, H2D inside)"})
     return latency
 
@@ -309,16 +342,111 @@ def staggered_run(ctx, states, host_ring, K, R, n_frames, window_ns, seed):
 
 
 # -------------------------------------------------------------------------------- GPU arm
+def stage_table(wl, K, stage_sum, steps, peaks):
+    """Per-stage device time, achieved rate and fraction of the roof that bounds the stage."""
+    stages = {}
+    for name, wk in stage_work(wl, K).items():
+        if name not in stage_sum:
+            continue
+        ms = stage_sum[name] / steps
+        ent = {"ms": ms, "bound": wk["bound"]}
+        if wk["bound"] == "hbm":
+            ent.update({"achieved": wk["bytes"] / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"})
+        elif wk["bound"] == "tensor":
+            ent.update({"achieved": wk["flops"] / (ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"})
+            ent["frac_of_sustained"] = ent["achieved"] / peaks["bf16_tflops_sustained"]
+        else:
+            ent.update({"achieved": wk["flops"] / (ms * 1e-3) / 1e12, "peak": FP32_ALU_TFLOPS, "unit": "TFLOP/s",
+                        "peak_source": "derived: 148 SMs x 128 fp32 FMA lanes x 2 x 1.965 GHz (not measured)"})
+        ent["frac"] = ent["achieved"] / ent["peak"]
+        stages[name] = ent
+    return stages
+
+
+class Rig:
+    """One context with K streams of a workload, its frame rings and the L2 flush buffer."""
+
+    def __init__(self, wl, K, dev, local_rank, stream, ring, stream_ids, flush, host_frames=True):
+        import torch
+
+        import tt_synth
+        from paper_2402_04466_b200 import binding
+        self.wl, self.K, self.R, self.stream, self.flush = wl, K, ring, stream, flush
+        self.weights = tt_synth.make_weights(wl)
+        self.ctx = binding.Context(binding.make_config(wl, max_streams=K, device=local_rank, cuda_stream=stream.cuda_stream), self.weights)
+        self.states = [self.ctx.state_create() for _ in range(K)]
+        frames = [[torch.from_numpy(tt_synth.make_frame(wl.frame_kind, wl.stream_seed(sid), t, wl.src_w, wl.src_h)) for t in range(ring)]
+                  for sid in stream_ids]
+        self.host_ring = [[f.pin_memory() for f in fs] for fs in frames] if host_frames else None
+        self.dev_ring = [[f.to(dev) for f in fs] for fs in frames]
+
+    def flush_l2(self, i):
+        import torch
+        with torch.cuda.stream(self.stream):
+            self.flush.fill_(i & 0xFF)
+
+    def tick(self, i, ring, K=None):
+        K = K or self.K
+        self.ctx.submit_frames([ring[s][i % self.R] for s in range(K)], self.states[:K], frame_index=i)
+        return self.ctx.sync()
+
+    def timed_ticks(self, steps, warmup):
+        """-> summed device time (ms) of `steps` ticks on device-resident frames, L2 flushed before each."""
+        for i in range(warmup):
+            self.flush_l2(i)
+            self.tick(i, self.dev_ring)
+        ms = []
+        for i in range(steps):
+            self.flush_l2(i)
+            ms.append(self.tick(i, self.dev_ring)[0]["gpu_ms"])
+        return ms
+
+    def stage_ticks(self, steps):
+        """The same ticks with an event recorded after every stage -> summed stage times, summed tick time."""
+        self.ctx.set_profiling(True)
+        stage_sum, prof_ms = {}, 0.0
+        for i in range(steps):
+            self.flush_l2(i)
+            res = self.tick(i, self.dev_ring)
+            prof_ms += res[0]["gpu_ms"]
+            for k, v in self.ctx.get_stage_times().items():
+                stage_sum[k] = stage_sum.get(k, 0.0) + v
+        self.ctx.set_profiling(False)
+        return stage_sum, prof_ms
+
+    def reset(self):
+        for s in self.states:
+            self.ctx.state_reset(s)
+
+    def destroy(self):
+        self.ctx.destroy()
+
+
+def stream_sweep(rig_of, counts, steps, warmup, paced_frames):
+    """frames/s and paced latency for several stream counts; rig_of(K) -> a Rig with at least K streams' frames."""
+    out = []
+    for Ks in counts:
+        rig = rig_of(Ks)
+        ms = rig.timed_ticks(steps, warmup)
+        ent = {"streams": Ks, "frames_per_s": Ks * len(ms) / (sum(ms) * 1e-3), "ms_per_tick": sum(ms) / len(ms)}
+        if paced_frames > 0:
+            rig.reset()
+            lat = paced_run(rig.ctx, rig.states, rig.host_ring, Ks, rig.R, paced_frames)
+            ent.update({k: lat[k] for k in ("p50_ms", "p99_ms", "max_ms", "spread_p99_p50_ms", "flatness_p90_p10_ms",
+                                            "tail_p100_p95_ms", "deadline_misses", "gpu_ms_mean")})
+        out.append(ent)
+        rig.destroy()
+    return out
+
+
 def run_ours(args):
     import ctypes as C
 
-    import numpy as np
     import torch
     import torch.distributed as dist
 
     import tt_synth
-    from paper_2402_04466_b200 import binding
-    from paper_2402_04466_b200.stats import latency_summary, trim_warmup
+    from paper_2402_04466_b200 import binding, sharding
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -340,31 +468,19 @@ def run_ours(args):
     K = args.streams or wl.streams
     if args.overlay is not None:
         wl = wl.with_(overlay=bool(args.overlay))
-    weights = tt_synth.make_weights(wl)
     stream = torch.cuda.Stream()
-    cfg = binding.make_config(wl, max_streams=K, device=local_rank, cuda_stream=stream.cuda_stream)
-    ctx = binding.Context(cfg, weights)
-    states = [ctx.state_create() for _ in range(K)]
-
-    # ring of distinct frames per stream (seeded; stream s of rank r uses seed index r*K + s)
-    R = args.ring
-    host_ring = [[torch.from_numpy(tt_synth.make_frame(wl.frame_kind, wl.stream_seed(rank * K + s), t, wl.src_w, wl.src_h)).pin_memory()
-                  for t in range(R)] for s in range(K)]
-    dev_ring = [[f.to(dev) for f in host_ring[s]] for s in range(K)]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    # Streams are independent problems: the world*K streams of the job are dealt round-robin to the ranks
+    # (stream s lives on rank s mod world), each rank runs its K streams, nothing is exchanged on the GPU.
+    my_streams = sharding.assign_streams(world * K, world)[rank]
+    R = args.ring
+    rig = Rig(wl, K, dev, local_rank, stream, R, my_streams, flush)
+    ctx, states, host_ring, dev_ring = rig.ctx, rig.states, rig.host_ring, rig.dev_ring
     frame_bytes = wl.src_h * wl.src_pitch
 
-    def tick(i, ring):
-        ctx.submit_frames([ring[s][i % R] for s in range(K)], states, frame_index=i)
-        return ctx.sync()
-
-    def flush_l2(i):
-        with torch.cuda.stream(stream):
-            flush.fill_(i & 0xFF)
-
     for i in range(args.warmup):
-        flush_l2(i)
-        tick(i, dev_ring)
+        rig.flush_l2(i)
+        rig.tick(i, dev_ring)
 
     uuid = None
     try:
@@ -376,99 +492,136 @@ def run_ours(args):
 
     # ---- timed region 1: device-resident frames, device time per tick from CUDA events
     barrier()
-    step_ms = []
-    for i in range(args.steps):
-        flush_l2(i)
-        res = tick(i, dev_ring)
-        step_ms.append(res[0]["gpu_ms"])
+    step_ms = rig.timed_ticks(args.steps, 0)
     barrier()
     launches1, _ = ctx.get_counters()
     total_ms = float(sum(step_ms))
 
     # ---- the same K steps again with an event recorded after every stage (per-kernel durations for
     # the roofline figures; the extra event records cost a few percent, so `value` comes from above)
-    ctx.set_profiling(True)
-    stage_sum, prof_ms = {}, 0.0
-    for i in range(args.steps):
-        flush_l2(i)
-        res = tick(i, dev_ring)
-        prof_ms += res[0]["gpu_ms"]
-        for k, v in ctx.get_stage_times().items():
-            stage_sum[k] = stage_sum.get(k, 0.0) + v
-    ctx.set_profiling(False)
+    stage_sum, prof_ms = rig.stage_ticks(args.steps)
     barrier()
 
     # ---- timed region 2: end to end through the public calls with pinned host frames.
     # (a) one tick at a time: submit -> sync, L2 flushed outside the timed part;
     # (b) software-pipelined, the way a throughput-oriented caller drives the API: tick i+1 is
     #     submitted before tick i is synced, so its host->device copy overlaps tick i's compute.
-    #     The L2 flush stays in stream order between ticks and its time counts against the number.
+    #     Once without any flush (every step's input crosses PCIe from host memory, so no cache can
+    #     hold it; weights and activations stay where a running service would have them), once with
+    #     the 256 MiB flush write in stream order between ticks, whose time then counts against the number.
     barrier()
     e2e_serial_s = 0.0
     for i in range(args.steps):
-        flush_l2(i)
+        rig.flush_l2(i)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        tick(i, host_ring)
+        rig.tick(i, host_ring)
         e2e_serial_s += time.perf_counter() - t0
     barrier()
-    t0 = time.perf_counter()
-    flush_l2(0)
-    ctx.submit_frames([host_ring[s][0] for s in range(K)], states, frame_index=0)
-    for i in range(1, args.steps):
-        flush_l2(i)
-        ctx.submit_frames([host_ring[s][i % R] for s in range(K)], states, frame_index=i)
-        ctx.sync()
-    ctx.sync()
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    barrier()
-    clocks = sampler.stop() if sampler else None
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_s, e2e_serial_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_s, e2e_serial_s = float(t[0]), float(t[1]), float(t[2])
+    def pipelined(with_flush):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        if with_flush:
+            rig.flush_l2(0)
+        ctx.submit_frames([host_ring[s][0] for s in range(K)], states, frame_index=0)
+        for i in range(1, args.steps):
+            if with_flush:
+                rig.flush_l2(i)
+            ctx.submit_frames([host_ring[s][i % R] for s in range(K)], states, frame_index=i)
+            ctx.sync()
+        last = ctx.sync()
+        torch.cuda.synchronize()
+        return time.perf_counter() - t0, last
+
+    e2e_s, last_results = pipelined(False)
+    barrier()
+    e2e_flush_s, _ = pipelined(True)
+    barrier()
+
+    total_ms, e2e_s, e2e_serial_s, e2e_flush_s = sharding.max_over_ranks([total_ms, e2e_s, e2e_serial_s, e2e_flush_s], world, device=dev)
+    # host-side gather of the small per-frame result records of the last tick (the only cross-rank data)
+    local = {sid: {"conf": [float(v) for v in r["conf"]], "count": [int(v) for v in r["count"]]} for sid, r in zip(my_streams, last_results)}
+    gathered = sharding.gather_results(local, world)
+    if len(gathered) != world * K:
+        raise RuntimeError(f"gathered {len(gathered)} result records, expected {world * K}")
 
     # ---- paced latency run (rank 0 of a single-GPU job): frames arrive every 16.7 ms per stream
     latency = None
     if world == 1 and args.paced_frames > 0:
-        for s in states:
-            ctx.state_reset(s)
+        rig.reset()
         latency = paced_run(ctx, states, host_ring, K, R, args.paced_frames)
 
     staggered = None
     if world == 1 and args.staggered_frames > 0:
-        for s in states:
-            ctx.state_reset(s)
+        rig.reset()
         staggered = staggered_run(ctx, states, host_ring, K, R, args.staggered_frames, int(args.window_ms * 1e6), wl.seed)
 
-    # ---- optional sweep over the number of streams (spec report: K = 1..8)
+    # the sampler covers the timed regions and the paced runs (a 20-step timed region alone lasts a few ms)
+    clocks_main = sampler.stop() if sampler else None
+
+    # ---- optional sweep over the number of streams of this workload
     sweep = None
     if world == 1 and args.sweep:
-        sweep = []
-        for Ks in [int(x) for x in args.sweep.split(",")]:
-            wls = wl
-            ctx_s = binding.Context(binding.make_config(wls, max_streams=Ks, device=local_rank, cuda_stream=stream.cuda_stream), weights)
-            st_s = [ctx_s.state_create() for _ in range(Ks)]
-            ring_h = [host_ring[s % K] for s in range(Ks)]
-            ring_d = [dev_ring[s % K] for s in range(Ks)]
-            ms = []
-            for i in range(args.warmup + args.sweep_steps):
-                flush_l2(i)
-                ctx_s.submit_frames([ring_d[s][i % R] for s in range(Ks)], st_s, frame_index=i)
-                r = ctx_s.sync()
-                if i >= args.warmup:
-                    ms.append(r[0]["gpu_ms"])
-            ent = {"streams": Ks, "frames_per_s": Ks * len(ms) / (sum(ms) * 1e-3), "ms_per_tick": sum(ms) / len(ms)}
-            if args.sweep_paced_frames > 0:
-                for s_ in st_s:
-                    ctx_s.state_reset(s_)
-                lat = paced_run(ctx_s, st_s, ring_h, Ks, R, args.sweep_paced_frames)
-                ent.update({k: lat[k] for k in ("p50_ms", "p99_ms", "max_ms", "spread_p99_p50_ms", "flatness_p90_p10_ms",
-                                                "tail_p100_p95_ms", "deadline_misses", "gpu_ms_mean")})
-            sweep.append(ent)
-            ctx_s.destroy()
+        counts = [int(x) for x in args.sweep.split(",")]
+        sweep = stream_sweep(lambda Ks: Rig(wl, Ks, dev, local_rank, stream, R, [my_streams[s % K] for s in range(Ks)], flush),
+                             counts, args.sweep_steps, args.warmup, args.sweep_paced_frames)
+
+    peaks, peak_kind = load_peaks()
+
+    # ---- the configuration the roofline targets are stated on (scale sweep, K = 8) and the stream-count
+    # sweeps of both sizes, in the same process
+    target = None
+    if world == 1 and args.target_steps > 0 and not (wl.name == "cfg4" and K == 8):
+        sampler_t = ClockSampler(uuid)
+        wt = tt_synth.workload("cfg4")
+        Kt = wt.streams
+        rig_t = Rig(wt, Kt, dev, local_rank, stream, 2, [s for s in range(Kt)], flush, host_frames=True)
+        ms_t = rig_t.timed_ticks(args.target_steps, args.warmup)
+        stage_t, prof_t = rig_t.stage_ticks(args.target_steps)
+        stages_t = stage_table(wt, Kt, stage_t, args.target_steps, peaks)
+        target = {"workload": describe(wt, Kt), "steps": args.target_steps, "warmup": args.warmup,
+                  "ms_per_step": sum(ms_t) / len(ms_t), "value": Kt * len(ms_t) / (sum(ms_t) * 1e-3), "unit": UNIT,
+                  "ms_per_step_with_stage_events": prof_t / args.target_steps, "stages": stages_t,
+                  "peaks": "tensor stages: frac against the measured burst bf16 peak, frac_of_sustained against the sustained one "
+                           "(the tick runs under the power cap); hbm stages against the measured copy bandwidth"}
+        if args.target_sweeps:
+            rig_t.reset()
+            sw4 = []
+            for Ks in (1, 2, 4, 8):
+                # one context sized for 8 streams serves every K: a tick of the first Ks streams
+                ms = []
+                for i in range(args.warmup + args.target_steps):
+                    rig_t.flush_l2(i)
+                    r = rig_t.tick(i, rig_t.dev_ring, Ks)
+                    if i >= args.warmup:
+                        ms.append(r[0]["gpu_ms"])
+                rig_t.reset()
+                lat = paced_run(rig_t.ctx, rig_t.states[:Ks], rig_t.host_ring, Ks, rig_t.R, args.target_paced_frames)
+                sw4.append({"streams": Ks, "frames_per_s": Ks * len(ms) / (sum(ms) * 1e-3), "ms_per_tick": sum(ms) / len(ms),
+                            "p50_ms": lat["p50_ms"], "p99_ms": lat["p99_ms"], "max_ms": lat["max_ms"],
+                            "flatness_p90_p10_ms": lat["flatness_p90_p10_ms"], "deadline_misses": lat["deadline_misses"]})
+            target["sweep_cfg4"] = sw4
+        rig_t.destroy()
+        if args.target_sweeps:
+            sw2 = []
+            w2 = tt_synth.workload("cfg2")
+            rig_2 = Rig(w2, 8, dev, local_rank, stream, R, list(range(8)), flush)
+            for Ks in range(1, 9):
+                ms = []
+                for i in range(args.warmup + 3 * args.target_steps):
+                    rig_2.flush_l2(i)
+                    r = rig_2.tick(i, rig_2.dev_ring, Ks)
+                    if i >= args.warmup:
+                        ms.append(r[0]["gpu_ms"])
+                rig_2.reset()
+                lat = paced_run(rig_2.ctx, rig_2.states[:Ks], rig_2.host_ring, Ks, rig_2.R, args.target_paced_frames)
+                sw2.append({"streams": Ks, "frames_per_s": Ks * len(ms) / (sum(ms) * 1e-3), "ms_per_tick": sum(ms) / len(ms),
+                            "p50_ms": lat["p50_ms"], "p99_ms": lat["p99_ms"], "max_ms": lat["max_ms"],
+                            "flatness_p90_p10_ms": lat["flatness_p90_p10_ms"], "deadline_misses": lat["deadline_misses"]})
+            rig_2.destroy()
+            target["sweep_cfg2"] = sw2
+        target["clocks"] = sampler_t.stop()
 
     if rank != 0:
         ctx.destroy()
@@ -476,27 +629,14 @@ def run_ours(args):
             dist.destroy_process_group()
         return 0
 
-    peaks, peak_kind = load_peaks()
-    work = stage_work(wl, K)
-    stages = {}
-    for name, wk in work.items():
-        if name not in stage_sum:
-            continue
-        ms = stage_sum[name] / args.steps
-        ent = {"ms": ms, "bound": wk["bound"]}
-        if wk["bound"] == "hbm":
-            ent.update({"achieved": wk["bytes"] / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"})
-        elif wk["bound"] == "tensor":
-            ent.update({"achieved": wk["flops"] / (ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"})
-        else:
-            ent.update({"achieved": wk["flops"] / (ms * 1e-3) / 1e12, "peak": None, "unit": "TFLOP/s"})
-        ent["frac"] = ent["achieved"] / ent["peak"] if ent.get("peak") else None
-        stages[name] = ent
+    stages = stage_table(wl, K, stage_sum, args.steps, peaks)
     dom = max(stages, key=lambda n: stages[n]["ms"])
     d = stages[dom]
     roofline = {"kernel": dom, "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"], "unit": d["unit"],
                 "frac": d["frac"], "traffic": recorded_traffic(dom, wl.name.replace("-gain", ""), K), "peak_source": f"of {peak_kind} (burst figure)",
                 "launch_ms": d["ms"]}
+    if "frac_of_sustained" in d:
+        roofline["frac_of_sustained"] = d["frac_of_sustained"]
 
     cpu_baseline = time_oracle(wl.with_(overlay=False)) if (world == 1 and not args.no_cpu_baseline) else None
     n_frames = world * K * args.steps
@@ -505,16 +645,19 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "ms_per_step_with_stage_events": prof_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if wl.precision == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": describe(wl, K), "streams_per_gpu": K, "frame_ring": R,
+                   "sharding": "stream s of the job on rank s mod N; no data-path collective; host-side gather of the result records",
                    "l2": "flushed between timed steps (256 MiB device write outside the timed events)",
                    "timing": "CUDA events on the launching stream around every tick, summed over the timed steps"},
         "e2e": {"value": n_frames / e2e_s, "unit": UNIT, "h2d_bytes_per_step": K * frame_bytes,
                 "d2h_bytes_per_step": K * C.sizeof(binding.tt_result) + 4,
+                "value_with_l2_flush": n_frames / e2e_flush_s,
                 "serial_value": n_frames / e2e_serial_s,
-                "timing": "host clock, pinned host frames; value: two submits in flight (tick i+1 submitted before tick i is "
-                          "synced), L2 flush between ticks included; serial_value: submit -> sync one tick at a time, "
-                          "flush outside the timed part"},
+                "timing": "host clock, pinned host frames, host->device copies and the device->host result read inside. value: two "
+                          "submits in flight (tick i+1 submitted before tick i is synced), no cache flush (each step's input comes "
+                          "from host memory); value_with_l2_flush: the same with a 256 MiB flush write in stream order between ticks, "
+                          "its time included; serial_value: submit -> sync one tick at a time, flush outside the timed part"},
         "gpu_launches": launches1 - launches0,
-        "roofline": roofline, "stages": stages, "clocks": clocks,
+        "roofline": roofline, "stages": stages, "clocks": clocks_main,
     }
     if latency is not None:
         line["latency"] = latency
@@ -522,6 +665,8 @@ def run_ours(args):
         line["latency_staggered"] = staggered
     if sweep is not None:
         line["sweep"] = sweep
+    if target is not None:
+        line["target_config"] = target
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline
     print(json.dumps(line))
@@ -542,13 +687,17 @@ def main():
     ap.add_argument("--overlay", type=int, default=None)
     ap.add_argument("--ring", type=int, default=8, help="distinct frames per stream, reused cyclically")
     ap.add_argument("--paced-frames", type=int, default=600, help="frames per stream of the paced latency run (0: skip)")
-    ap.add_argument("--staggered-frames", type=int, default=0,
+    ap.add_argument("--staggered-frames", type=int, default=300,
                     help="frames per stream of the unsynchronised-arrival run through the batch planner (0: skip)")
     ap.add_argument("--window-ms", type=float, default=1.0, help="coalescing window of the batch planner")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", default="", help="comma-separated stream counts to measure in addition, e.g. 1,2,3,4,5,6,7,8")
     ap.add_argument("--sweep-steps", type=int, default=100)
     ap.add_argument("--sweep-paced-frames", type=int, default=200)
+    ap.add_argument("--target-steps", type=int, default=10,
+                    help="timed ticks of the scale-sweep configuration (cfg4, K=8) reported as target_config (0: skip)")
+    ap.add_argument("--target-sweeps", type=int, default=1, help="also sweep the stream count at both sizes (0: skip)")
+    ap.add_argument("--target-paced-frames", type=int, default=120, help="frames per stream of every sweep point's paced run")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

@@ -569,7 +569,7 @@ def test_staggered_arrivals_through_the_planner_match_per_stream_runs(cuda_devic
     sids = [sched.admit() for _ in range(K)]
     phases = [0, 100_000, 200_000, 9 * ms]                        # streams 1, 2 arrive while stream 0's tick is in flight
     arrivals = sorted((phases[k] + t * period + (23_000 * ((t * 7 + k) % 5)), k, t) for k in range(K) for t in range(n))
-    ctx, states, _ = _make(wl, K)
+    ctx, states, w_ = _make(wl, K)
     got = {}
     sizes = []
     pending = list(arrivals)
@@ -598,6 +598,14 @@ def test_staggered_arrivals_through_the_planner_match_per_stream_runs(cuda_devic
     assert st["frames"] == K * n and st["dropped"] == 0 and st["deadline_misses"] == 0
     assert len(got) == K * n and min(sizes) == 1 and max(sizes) >= 2 and st["batches"] < K * n
     ctx.destroy()
+    # one of the staggered streams against the oracle, frame by frame: whatever batches its frames shared, the
+    # stream must be the oracle's stream (each side carrying its own recurrent state through all n frames)
+    ora = oracle.OraclePipeline(wl, w_)
+    for t in range(n):
+        ref = ora.step(frames[2][t], want_overlay=False)
+        p, conf, cnt, cx = got[(2, t)]
+        assert_close(p, ref.p, TOL_OUT, f"staggered stream 2 t={t} prob")
+        assert_close(conf, ref.conf, TOL_OUT, f"staggered stream 2 t={t} conf")
     ctx1, (s1,), _ = _make(wl, 1)
     for k in range(K):
         ctx1.state_reset(s1)
