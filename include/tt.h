@@ -82,7 +82,8 @@ typedef struct {
   float threshold;                 /* on the sigmoid, in (0,1) */
   int32_t overlay;                 /* non-zero: also produce the RGBA8 overlay per frame */
   uint8_t palette[TT_MAX_TOOLS][3];
-  uint8_t reserved_[8];            /* reserved_[0] != 0: launch every tick as plain kernel launches, never from a CUDA graph */
+  uint8_t reserved_[8];            /* reserved_[0] != 0: launch every tick as plain kernel launches, never from a CUDA graph;
+                                      reserved_[2] != 0: never run tensor-core layers on CTA pairs (for A/B measurements) */
   void* cuda_stream;               /* cudaStream_t owned by the caller, or NULL: the library creates one */
   uint64_t sync_timeout_ns;        /* 0: wait without limit in tt_sync */
 } tt_config;

@@ -149,7 +149,7 @@ def _check(lib, status: int, ctx=None):
 
 def make_config(wl, max_streams: int = 1, device: int = 0, overlay: Optional[bool] = None,
                 cuda_stream: int = 0, sync_timeout_ns: int = 0, precision: Optional[str] = None,
-                plain_launches: bool = False) -> tt_config:
+                plain_launches: bool = False, cta_pairs: bool = True) -> tt_config:
     """Fill a tt_config from any object carrying the workload attributes (src_w, net_w, enc_cout, ...).
 
     plain_launches=True makes every tick launch its kernels one by one instead of replaying a CUDA graph."""
@@ -177,6 +177,7 @@ def make_config(wl, max_streams: int = 1, device: int = 0, overlay: Optional[boo
     cfg.cuda_stream = cuda_stream or None
     cfg.sync_timeout_ns = sync_timeout_ns
     cfg.reserved_[0] = 1 if plain_launches else 0
+    cfg.reserved_[2] = 0 if cta_pairs else 1
     return cfg
 
 

@@ -41,10 +41,14 @@ constexpr int EPI_WARP0 = 2;
 constexpr int TC_THREADS = 32 * (2 + EPI_WARPS + (N_PROD - 1));
 constexpr int MAX_K_ITERS = 9 * 16;                // 9 taps x up to 16 channel slabs
 
-template <int BLOCK_N, int SLAB_C>
+// PAIR: two CTAs of a cluster work on two neighbouring M-tiles with one MMA of 256 rows
+// (cta_group::2).  Each CTA then stages its own activation box and only its own half of the
+// weight slab's rows, so a stage holds a third less and the ring is half as deep again.
+template <int BLOCK_N, int SLAB_C, bool PAIR = false>
 struct TcCfg {
   static constexpr int A_BYTES = BLOCK_M * SLAB_C * 2;
-  static constexpr int B_BYTES = BLOCK_N * SLAB_C * 2;
+  static constexpr int B_ROWS = PAIR ? BLOCK_N / 2 : BLOCK_N;     // weight rows staged by one CTA
+  static constexpr int B_BYTES = B_ROWS * SLAB_C * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES_RAW = (192 * 1024) / STAGE_BYTES;
   static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
@@ -68,13 +72,13 @@ __device__ __forceinline__ float fast_sigmoid(float z) { return fmaf(0.5f, fast_
 
 
 // ------------------------------------------------------------------------------------ kernel
-template <int BLOCK_N, int SLAB_C, int EPI>
+template <int BLOCK_N, int SLAB_C, int EPI, bool PAIR>
 __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_constant__ ConvTcParams p) {
-  using Cfg = TcCfg<BLOCK_N, SLAB_C>;
+  using Cfg = TcCfg<BLOCK_N, SLAB_C, PAIR>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr uint32_t LAYOUT = SLAB_C == 64 ? 2u : 4u;
   constexpr uint32_t SBO = 8u * SLAB_C * 2u;
-  constexpr uint32_t IDESC = make_idesc(BLOCK_M, BLOCK_N);
+  constexpr uint32_t IDESC = make_idesc(PAIR ? 2 * BLOCK_M : BLOCK_M, BLOCK_N);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -92,7 +96,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wait_limit = p.wait_limit;
   const int tiles_per_img = p.tiles_x * p.tiles_y;
-  const int total_tiles = p.K * tiles_per_img * p.n_tiles_n;
+  // Units of work: a tile (M-tile x N-tile), or for a CTA pair two neighbouring M-tiles x N-tile.
+  // `worker` counts CTAs (or pairs), `rank` is this CTA's place in its pair, `m_tiles` the M-tiles.
+  const int m_tiles = p.K * tiles_per_img;
+  const int total_tiles = (PAIR ? (m_tiles + 1) / 2 : m_tiles) * p.n_tiles_n;
+  const int rank = PAIR ? (int)cluster_ctarank() : 0;
+  const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const int slabs_per_tap = p.slabs[0] + (p.n_src > 1 ? p.slabs[1] : 0);
   const int k_iters = 9 * slabs_per_tap;
 
@@ -126,13 +136,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
   }
 
   if (threadIdx.x == 0) {
+    // in a pair the leader's "full" barriers collect one arrival per CTA and the bytes of both
+    // CTAs' copies; its "accumulator free" barriers collect the epilogue warps of both CTAs
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(smem_u32(full_bar + s), 1);
+      mbar_init(smem_u32(full_bar + s), PAIR ? 2 : 1);
       mbar_init(smem_u32(empty_bar + s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(tfull_bar + a), 1);
-      mbar_init(smem_u32(tempty_bar + a), EPI_WARPS);
+      mbar_init(smem_u32(tempty_bar + a), PAIR ? 2 * EPI_WARPS : EPI_WARPS);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -140,13 +152,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
   }
   if (warp == MMA_WARP) {
     __syncwarp();   // the table loop above may have left the warp's lanes apart; the allocation is warp-collective
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"((uint32_t)Cfg::TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (PAIR) {
+      // the same warp of both CTAs allocates the pair's columns
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"((uint32_t)Cfg::TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"((uint32_t)Cfg::TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // the peer's barriers exist before anything is signalled across the pair
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();   // everything above touched no activation; from here on the previous kernel's outputs are read
@@ -161,9 +182,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     int it = prod;
     bool ok = true;
     const uint8_t* maps = reinterpret_cast<const uint8_t*>(p.maps_a);
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+    // a pair's copies are counted on the leader's barriers
+    const uint32_t full0c = PAIR ? map_to_cta(smem_u32(full_bar), 0u) : 0u;
+    for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
       const int nt = tile % p.n_tiles_n;
-      const int m = tile / p.n_tiles_n;
+      // the second CTA of a pair takes the next M-tile; past the end it recomputes the last one (its epilogue stores nothing)
+      const int m = PAIR ? min(2 * (tile / p.n_tiles_n) + rank, m_tiles - 1) : tile / p.n_tiles_n;
       const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
       const int x0 = tx * PATCH_W, y0 = ty * PATCH_H;
       // (two scalars, not an indexed array: an array would live in local memory, and a memory round
@@ -173,17 +197,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
         const int4 e = s_tab[it];
         ok = mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag, p.status, 0x100 + (int)stage, wait_limit);
         if (!ok) break;
-        const uint32_t fb = smem_u32(full_bar + stage);
         uint8_t* st = smem + stage * Cfg::STAGE_BYTES;
-        mbar_arrive_expect_tx(fb, Cfg::STAGE_BYTES);
-        tma_load_4d(smem_u32(st), maps + e.x * (int)sizeof(TensorMap128), fb, e.y, x0 + e.z, y0 + e.w, e.x < 4 ? img_x : img_h);
-        tma_load_2d(smem_u32(st + Cfg::A_BYTES), &p.map_b, fb, it * SLAB_C, nt * BLOCK_N);
+        if (PAIR) {
+          const uint32_t fb = full0c + 8u * stage;
+          mbar_arrive_expect_tx_cluster(fb, Cfg::STAGE_BYTES);
+          tma_load_4d_pair(smem_u32(st), maps + e.x * (int)sizeof(TensorMap128), fb, e.y, x0 + e.z, y0 + e.w, e.x < 4 ? img_x : img_h);
+          tma_load_2d_pair(smem_u32(st + Cfg::A_BYTES), &p.map_b, fb, it * SLAB_C, nt * BLOCK_N + rank * Cfg::B_ROWS);
+        } else {
+          const uint32_t fb = smem_u32(full_bar + stage);
+          mbar_arrive_expect_tx(fb, Cfg::STAGE_BYTES);
+          tma_load_4d(smem_u32(st), maps + e.x * (int)sizeof(TensorMap128), fb, e.y, x0 + e.z, y0 + e.w, e.x < 4 ? img_x : img_h);
+          tma_load_2d(smem_u32(st + Cfg::A_BYTES), &p.map_b, fb, it * SLAB_C, nt * BLOCK_N);
+        }
         stage += (uint32_t)n_prod;
         if (stage >= (uint32_t)STAGES) { stage -= STAGES; phase ^= 1u; }
       }
       it -= k_iters;
     }
-  } else if (warp == MMA_WARP && lane == 0) {
+  } else if (warp == MMA_WARP && lane == 0 && rank == 0) {
     // -------------------------------------------------------------------- MMA issuer
     // This loop is one thread's chain of dependent instructions and sets the pace of the whole
     // block, so everything that does not change is formed once: the operand descriptors differ
@@ -196,7 +227,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     constexpr uint64_t STAGE_UNITS = Cfg::STAGE_BYTES >> 4, B_UNITS = Cfg::A_BYTES >> 4;
     const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
     uint64_t a_desc = a_desc0;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+    for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
       ok = mbar_wait(smem_u32(tempty_bar + acc), acc_phase ^ 1u, abort_flag, p.status, 0x200 + acc, wait_limit);
       if (!ok) break;
       tc_fence_after();   // the epilogue's TMEM reads of this buffer come before the MMAs that overwrite it
@@ -207,15 +238,23 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
         if (!ok) break;
         const uint64_t b_desc = a_desc + B_UNITS;
         // advance along K inside the swizzle atom: 16 bf16 = 32 bytes = 2 descriptor units
-        umma_bf16(d_tmem, a_desc, b_desc, IDESC, it != 0 ? 1u : 0u);
+        if (PAIR) {
+          umma_bf16_pair(d_tmem, a_desc, b_desc, IDESC, it != 0 ? 1u : 0u);
 #pragma unroll
-        for (int k = 1; k < SLAB_C / UMMA_K; ++k) umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), IDESC, 1u);
-        umma_commit(empty0 + 8u * stage);            // frees the stage once the MMAs have read it
+          for (int k = 1; k < SLAB_C / UMMA_K; ++k) umma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), IDESC, 1u);
+          umma_commit_pair(empty0 + 8u * stage);     // frees the stage in both CTAs once the MMAs have read it
+        } else {
+          umma_bf16(d_tmem, a_desc, b_desc, IDESC, it != 0 ? 1u : 0u);
+#pragma unroll
+          for (int k = 1; k < SLAB_C / UMMA_K; ++k) umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), IDESC, 1u);
+          umma_commit(empty0 + 8u * stage);          // frees the stage once the MMAs have read it
+        }
         a_desc += STAGE_UNITS;
         if (++stage == STAGES) { stage = 0; phase ^= 1u; a_desc = a_desc0; }
       }
       if (!ok) break;
-      umma_commit(smem_u32(tfull_bar + acc));      // accumulator complete
+      if (PAIR) umma_commit_pair(smem_u32(tfull_bar + acc));   // accumulator complete, in both CTAs
+      else umma_commit(smem_u32(tfull_bar + acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + EPI_WARPS) {
@@ -231,12 +270,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
     uint32_t acc_phase = 0;
     int acc = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    const uint32_t tempty0c = PAIR ? map_to_cta(smem_u32(tempty_bar), 0u) : 0u;
+    for (int tile = worker; tile < total_tiles; tile += n_workers) {
       const int nt = tile % p.n_tiles_n;
-      const int m = tile / p.n_tiles_n;
+      const int m_raw = PAIR ? 2 * (tile / p.n_tiles_n) + rank : tile / p.n_tiles_n;
+      const int m = min(m_raw, m_tiles - 1);
       const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
       const int x = tx * PATCH_W + px, y = ty * PATCH_H + py;
-      const bool valid = x < p.Wo && y < p.Ho;
+      const bool valid = x < p.Wo && y < p.Ho && m_raw < m_tiles;
       const size_t pix = (size_t)y * p.Wo + x;
       const int col0 = nt * BLOCK_N + half * HALF_N;  // first packed output column of this warp
 
@@ -322,7 +363,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
       // hand the accumulator buffer back to the MMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(tempty_bar + acc));
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_cluster(tempty0c + 8u * (uint32_t)acc);
+        else mbar_arrive(smem_u32(tempty_bar + acc));
+      }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }
@@ -336,17 +380,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
   }
   tc_fence_before();
   __syncthreads();
+  // neither CTA of a pair may go while the other can still signal its barriers or have its shared memory read by the pair's MMAs
+  if (PAIR) cluster_sync_all();
   if (warp == MMA_WARP) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS)
-                 : "memory");
+    if (PAIR)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
   }
 }
 
 template <int BLOCK_N, int SLAB_C, int EPI>
 cudaError_t launch_cfg(const ConvTcParams& p, int sm_count, cudaStream_t s) {
   using Cfg = TcCfg<BLOCK_N, SLAB_C>;
-  auto kern = conv_tc_kernel<BLOCK_N, SLAB_C, EPI>;
+  auto kern = conv_tc_kernel<BLOCK_N, SLAB_C, EPI, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int total_tiles = p.K * p.tiles_x * p.tiles_y * p.n_tiles_n;
@@ -354,8 +402,49 @@ cudaError_t launch_cfg(const ConvTcParams& p, int sm_count, cudaStream_t s) {
   return launch_kernel(kern, grid, TC_THREADS, Cfg::SMEM_BYTES, s, p, p.pdl != 0);
 }
 
+// CTA pairs: clusters of two, one pair per unit of work, as many pairs as the device can hold at once.
+template <int BLOCK_N, int SLAB_C, int EPI>
+cudaError_t launch_pair(const ConvTcParams& p, int sm_count, cudaStream_t s) {
+  using Cfg = TcCfg<BLOCK_N, SLAB_C, true>;
+  auto kern = conv_tc_kernel<BLOCK_N, SLAB_C, EPI, true>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg{};
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.pdl ? 2 : 1;
+  // pairs that can be resident at once (a pair needs two multiprocessors of one cluster-capable group)
+  static int max_pairs = 0;   // the same for every instantiation's launch shape: one block per multiprocessor
+  if (max_pairs == 0) {
+    cfg.gridDim = dim3((unsigned)(2 * (sm_count / 2)));
+    int n = 0;
+    e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+    if (e != cudaSuccess) return e;
+    if (n < 1) return cudaErrorInvalidConfiguration;
+    max_pairs = n;
+  }
+  const int m_tiles = p.K * p.tiles_x * p.tiles_y;
+  const int units = ((m_tiles + 1) / 2) * p.n_tiles_n;
+  const int pairs = units < max_pairs ? units : max_pairs;
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
 template <int EPI>
 cudaError_t launch_shape(const ConvTcParams& p, int sm_count, cudaStream_t s) {
+  if (p.pair) {
+    if (p.slab_c == 64 && p.block_n == 256) return launch_pair<256, 64, EPI>(p, sm_count, s);
+    return cudaErrorInvalidValue;
+  }
   if (p.slab_c == 64) {
     if (p.block_n == 256) return launch_cfg<256, 64, EPI>(p, sm_count, s);
     if (p.block_n == 128) return launch_cfg<128, 64, EPI>(p, sm_count, s);

@@ -148,6 +148,7 @@ struct tt_ctx {
   };
   std::vector<TickGraph> graphs;
   bool graphs_off = false;
+  bool no_pairs = false;            // reserved_[2]: never run the tensor-core layers on CTA pairs
   const uint8_t** frame_tab_dev[2] = {nullptr, nullptr};   // device, [TT_MAX_STREAMS] pointers per slot
   const uint8_t** frame_tab_host[2] = {nullptr, nullptr};  // pinned staging of the same
   const uint8_t* const* cur_tab = nullptr;                  // table the tick being enqueued reads
@@ -497,6 +498,7 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
   }
   bind_slot(ctx, 0);
   ctx->graphs_off = c.reserved_[0] != 0;
+  ctx->no_pairs = c.reserved_[2] != 0;
 
   // ---- weights
   const bool r = ctx->bf16;  // round weights to bf16 on the bf16 path
@@ -689,6 +691,9 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
       if (bi < 0) return fail(ctx, TT_ERR_UNSUPPORTED, "no tensor-core tile shape fits this layer");
       const int bns[3] = {64, 128, 256};
       q.block_n = bns[bi]; q.map_b = L.map_b[bi]; q.n_tiles_n = L.cout / q.block_n;
+      // 256-wide tiles run on CTA pairs: each CTA stages its own activation box and half of the weight slab
+      q.pair = (bi == 2 && L.slab_c == 64 && L.has_b[1] && !ctx->no_pairs && K * q.tiles_x * q.tiles_y >= 2) ? 1 : 0;
+      if (q.pair) q.map_b = L.map_b[1];
       q.cout = L.cout; q.bias = L.b; q.status = ctx->status_dev; q.wait_limit = ctx->wait_limit;
       q.n_prod = 3;
       q.pdl = ctx->profiling ? 0 : 1;

@@ -13,10 +13,10 @@ from parity_util import assert_close, check_masks, check_reductions_from_own_mas
 pytestmark = pytest.mark.gpu
 
 
-def _make(wl, K=1, overlay=None, precision=None, timeout_ns=0, plain_launches=False):
+def _make(wl, K=1, overlay=None, precision=None, timeout_ns=0, plain_launches=False, cta_pairs=True):
     weights = tt_synth.make_weights(wl)
     cfg = binding.make_config(wl, max_streams=K, overlay=overlay, precision=precision, sync_timeout_ns=timeout_ns,
-                              plain_launches=plain_launches)
+                              plain_launches=plain_launches, cta_pairs=cta_pairs)
     ctx = binding.Context(cfg, weights)
     states = [ctx.state_create() for _ in range(K)]
     return ctx, states, weights
@@ -222,6 +222,28 @@ def test_bf16_wide_channels_small_map(cuda_device):
     wl = tt_synth.workload("cfg4-gain").with_(name="bf16-wide", src_w=160, src_h=120, net_w=136, net_h=104)
     assert wl.map_hw() == (13, 17)
     _run_bf16(cuda_device, wl, 2, 2)
+
+
+def test_bf16_cta_pairs_with_an_odd_number_of_tiles(cuda_device):
+    """The 256-wide ConvLSTM tiles run on CTA pairs (two neighbouring 128-pixel tiles per MMA).  Three streams of
+    an 80x40 map give 75 tiles: the last pair has no second tile, its second CTA recomputes the last tile and
+    must store nothing.  Checked against the oracle, and bit for bit against the same context without pairs."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="bf16-pairs", src_w=854, src_h=320, net_w=640, net_h=320)
+    assert wl.map_hw() == (40, 80)
+    _run_bf16(cuda_device, wl, 3, 2)
+    K, n = 3, 2
+    frames = _frames(wl, K, n)
+    outs = []
+    for pairs in (True, False):
+        ctx, states, _ = _make(wl, K, cta_pairs=pairs)
+        for t in range(n):
+            ctx.submit_frames([torch.from_numpy(frames[k][t]).to(cuda_device) for k in range(K)], states, frame_index=t)
+            res = ctx.sync()
+        outs.append(([ctx.state_export(s) for s in states], [ctx.fetch_probs(r) for r in res]))
+        ctx.destroy()
+    for k in range(K):
+        assert np.array_equal(outs[0][0][k][0], outs[1][0][k][0]) and np.array_equal(outs[0][0][k][1], outs[1][0][k][1])
+        assert np.array_equal(outs[0][1][k], outs[1][1][k])
 
 
 def test_bf16_stride1_encoder_and_overlay(cuda_device):
