@@ -49,6 +49,21 @@ typedef enum {
 } tt_status;
 
 typedef enum { TT_FP32 = 0, TT_BF16 = 1 } tt_precision;
+/* Indices into tt_config.options; a non-zero byte switches the option on. */
+typedef enum {
+  TT_OPT_PLAIN_LAUNCHES = 0, /* launch every tick as plain kernel launches, never from a CUDA graph */
+  TT_OPT_FEED_FORWARD = 1,   /* the model has no recurrent cell: encoder -> mask/confidence heads (the paper's second
+                                workload class, a feed-forward segmentation network, Section V-B); `hidden` must equal the
+                                last encoder width, lstm_w/lstm_b are ignored, states carry nothing */
+  TT_OPT_CTA_PAIRS = 2,      /* run 256-wide tensor-core tiles on CTA pairs (cta_group::2).  Off by default: measured
+                                11-15 % slower than single-CTA tiles on the benchmark shapes */
+  TT_OPT_RESERVED_SMS = 4,   /* value = number of multiprocessors left free for another workload (at most half of the
+                                device): the persistent tensor-core and post-processing kernels size their grids for the
+                                rest.  With tt_render_layers' carved-out form this gives the visualisation load its own
+                                multiprocessors (the single-GPU isolation the paper leaves as future work, Section VIII) */
+  TT_OPT_NO_POST_TC = 3      /* bf16 path: post-process from the fp32 hidden state, not from its bf16 copy on the
+                                tensor cores (for A/B measurements; not available for feed-forward models) */
+} tt_option;
 typedef enum { TT_CONF_MEAN_SIGMOID = 0, TT_CONF_GAP_LINEAR = 1 } tt_conf_mode;
 
 /* Which intermediate tensor tt_debug_tensor copies out (always NCHW fp32 on the host). */
@@ -82,8 +97,7 @@ typedef struct {
   float threshold;                 /* on the sigmoid, in (0,1) */
   int32_t overlay;                 /* non-zero: also produce the RGBA8 overlay per frame */
   uint8_t palette[TT_MAX_TOOLS][3];
-  uint8_t reserved_[8];            /* reserved_[0] != 0: launch every tick as plain kernel launches, never from a CUDA graph;
-                                      reserved_[2] != 0: never run tensor-core layers on CTA pairs (for A/B measurements) */
+  uint8_t options[8];              /* indexed by tt_option; all zero = defaults */
   void* cuda_stream;               /* cudaStream_t owned by the caller, or NULL: the library creates one */
   uint64_t sync_timeout_ns;        /* 0: wait without limit in tt_sync */
 } tt_config;
@@ -369,6 +383,24 @@ tt_status tt_postprocess_static(const float* h_dev, int32_t channels_last, int32
 tt_status tt_overlay(const uint8_t* src_dev, int32_t K, int64_t src_frame_stride, int32_t src_w, int32_t src_h,
                      int32_t src_pitch, const uint8_t* masks_dev, int32_t n_tools, int32_t hm, int32_t wm,
                      const uint8_t* palette_host, uint8_t* dst_dev, void* cuda_stream);
+
+/*
+ * tt_render_layers — a scaled-up stand-in for the visualisation load.  The paper finds that the
+ * visualisation work sharing a GPU with the inference work is what spreads the latencies
+ * (Section VI) and names single-GPU isolation of the two as future work (Section VIII).  This
+ * call is the "graphics" side of that experiment in CUDA: a full-resolution blend of `layers`
+ * layers; layer l applies tt_overlay's blend with tool t drawn in palette colour (t + l) mod
+ * n_tools, on the result of layer l - 1.  Arguments as for tt_overlay.
+ * carve_ctas == 0: time-shared form, one block per 1024 pixels spread over the whole device.
+ * carve_ctas  > 0: carved-out form, that many blocks loop over the batch, each claiming 64 KB of
+ * shared memory so that the inference path's large blocks are not placed beside it; give the
+ * inference context TT_OPT_RESERVED_SMS = carve_ctas so that it leaves those multiprocessors free.
+ * The arithmetic per pixel does not depend on the mask values.
+ */
+tt_status tt_render_layers(const uint8_t* src_dev, int32_t K, int64_t src_frame_stride, int32_t src_w, int32_t src_h,
+                           int32_t src_pitch, const uint8_t* masks_dev, int32_t n_tools, int32_t hm, int32_t wm,
+                           const uint8_t* palette_host, int32_t layers, int32_t carve_ctas, uint8_t* dst_dev,
+                           void* cuda_stream);
 
 #ifdef __cplusplus
 }

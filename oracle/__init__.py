@@ -10,9 +10,9 @@ Whole-pipeline parity is unpinned by any published value (the paper prints no te
 each stage is pinned separately by tests/test_oracle_*.py.
 """
 from .stages import (preprocess, resize_axis, conv3x3, convlstm_step, head, conf_mean_sigmoid,
-                     conf_gap_linear, centroids, overlay, round_bf16, num_threads, set_threads)
+                     conf_gap_linear, centroids, overlay, render_layers, round_bf16, num_threads, set_threads)
 from .pipeline import OraclePipeline, FrameOutput
 
 __all__ = ["preprocess", "resize_axis", "conv3x3", "convlstm_step", "head", "conf_mean_sigmoid",
-           "conf_gap_linear", "centroids", "overlay", "round_bf16", "num_threads", "set_threads",
+           "conf_gap_linear", "centroids", "overlay", "render_layers", "round_bf16", "num_threads", "set_threads",
            "OraclePipeline", "FrameOutput"]

@@ -65,9 +65,14 @@ class OraclePipeline:
             if self.mirror:
                 a = S.round_bf16(a)
             enc.append(a)
-        h_in = S.round_bf16(self.h) if self.mirror else self.h
-        h2, c2 = S.convlstm_step(a, h_in, self.c, w["lstm_w"], w["lstm_b"])
-        self.h, self.c = h2, c2
+        if getattr(wl, "recurrent", True):
+            h_in = S.round_bf16(self.h) if self.mirror else self.h
+            h2, c2 = S.convlstm_step(a, h_in, self.c, w["lstm_w"], w["lstm_b"])
+            self.h, self.c = h2, c2
+        else:
+            # feed-forward model (the paper's second workload class, Section V-B): the heads read the
+            # last encoder output; there is no state to carry
+            h2, c2 = enc[-1], np.zeros_like(enc[-1])
         z, p, mask = S.head(h2, w["head_w"], w["head_b"], wl.threshold)
         if wl.conf_mode == "mean_sigmoid":
             conf = S.conf_mean_sigmoid(p)

@@ -148,6 +148,21 @@ def overlay(frame, mask, palette):
     return dst
 
 
+def render_layers(frame, mask, palette, layers: int):
+    """Multi-layer stand-in for the visualisation load: the S6 blend applied `layers` times in sequence, layer l
+    with the palette rotated by l (tool t takes colour (t + l) mod T), each layer on the previous layer's RGB."""
+    if layers < 1:
+        raise ValueError("layers >= 1 required")
+    T = np.asarray(mask).shape[0]
+    pal = [tuple(int(v) for v in c) for c in np.asarray(palette, dtype=np.uint8)[:T]]
+    rgb = np.ascontiguousarray(frame, dtype=np.uint8)
+    out = None
+    for l in range(layers):
+        out = overlay(rgb, mask, [pal[(t + l) % T] for t in range(T)])
+        rgb = np.ascontiguousarray(out[..., :3])
+    return out
+
+
 def round_bf16(a):
     out = np.array(a, dtype=np.float32, order="C", copy=True)
     _lib.ora_round_bf16(out.reshape(-1), out.size)

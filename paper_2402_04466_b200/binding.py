@@ -21,6 +21,7 @@ TT_OK = 0
 STATUS_NAMES = {0: "TT_OK", 1: "TT_ERR_INVALID_ARG", 2: "TT_ERR_UNSUPPORTED", 3: "TT_ERR_OOM", 4: "TT_ERR_CUDA",
                 5: "TT_ERR_ADMISSION", 6: "TT_ERR_NOT_READY", 7: "TT_ERR_TIMEOUT", 8: "TT_ERR_DEVICE_STATUS"}
 TT_FP32, TT_BF16 = 0, 1
+TT_OPT_PLAIN_LAUNCHES, TT_OPT_FEED_FORWARD, TT_OPT_CTA_PAIRS, TT_OPT_NO_POST_TC, TT_OPT_RESERVED_SMS = 0, 1, 2, 3, 4
 TT_CONF_MEAN_SIGMOID, TT_CONF_GAP_LINEAR = 0, 1
 TENSOR_IDS = {"pre": 0, "enc0": 1, "enc1": 2, "enc2": 3, "enc3": 4, "h": 8, "c": 9, "logits": 10, "prob": 11}
 
@@ -30,7 +31,7 @@ EXPORTED_SYMBOLS = [
     "tt_set_profiling", "tt_get_stage_times", "tt_get_counters", "tt_query", "tt_debug_expire_wait",
     "tt_sched_create", "tt_sched_destroy", "tt_sched_admit", "tt_sched_release", "tt_sched_arrive", "tt_sched_next",
     "tt_sched_complete", "tt_sched_predict_ms", "tt_sched_stats",
-    "tt_preprocess", "tt_postprocess_scratch_bytes", "tt_postprocess", "tt_postprocess_static", "tt_overlay",
+    "tt_preprocess", "tt_postprocess_scratch_bytes", "tt_postprocess", "tt_postprocess_static", "tt_overlay", "tt_render_layers",
 ]
 TT_POSTPROCESS_STATIC_SCRATCH_BYTES = 32 << 10
 STAGE_NAMES = ["h2d", "preprocess", "enc0", "enc1", "enc2", "enc3", "convlstm", "postprocess", "overlay"]
@@ -52,7 +53,7 @@ class tt_config(C.Structure):
         ("n_enc", C.c_int32), ("enc_cout", C.c_int32 * TT_MAX_ENC), ("enc_stride", C.c_int32 * TT_MAX_ENC),
         ("hidden", C.c_int32), ("n_tools", C.c_int32), ("precision", C.c_int32), ("conf_mode", C.c_int32),
         ("threshold", C.c_float), ("overlay", C.c_int32),
-        ("palette", (C.c_uint8 * 3) * TT_MAX_TOOLS), ("reserved_", C.c_uint8 * 8),
+        ("palette", (C.c_uint8 * 3) * TT_MAX_TOOLS), ("options", C.c_uint8 * 8),
         ("cuda_stream", C.c_void_p), ("sync_timeout_ns", C.c_uint64),
     ]
 
@@ -135,6 +136,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.tt_postprocess.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp, vp]
     lib.tt_postprocess_static.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp]
     lib.tt_overlay.argtypes = [vp, i32, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp]
+    lib.tt_render_layers.argtypes = [vp, i32, i64, i32, i32, i32, vp, i32, i32, i32, vp, i32, i32, vp, vp]
     for name in EXPORTED_SYMBOLS:
         getattr(lib, name)  # AttributeError here means the library does not export what tt.h declares
     _LIB = lib
@@ -149,7 +151,8 @@ def _check(lib, status: int, ctx=None):
 
 def make_config(wl, max_streams: int = 1, device: int = 0, overlay: Optional[bool] = None,
                 cuda_stream: int = 0, sync_timeout_ns: int = 0, precision: Optional[str] = None,
-                plain_launches: bool = False, cta_pairs: bool = True) -> tt_config:
+                plain_launches: bool = False, cta_pairs: bool = False, post_tc: bool = True,
+                reserved_sms: int = 0) -> tt_config:
     """Fill a tt_config from any object carrying the workload attributes (src_w, net_w, enc_cout, ...).
 
     plain_launches=True makes every tick launch its kernels one by one instead of replaying a CUDA graph."""
@@ -176,8 +179,11 @@ def make_config(wl, max_streams: int = 1, device: int = 0, overlay: Optional[boo
             cfg.palette[t][k] = wl.palette[t][k]
     cfg.cuda_stream = cuda_stream or None
     cfg.sync_timeout_ns = sync_timeout_ns
-    cfg.reserved_[0] = 1 if plain_launches else 0
-    cfg.reserved_[2] = 0 if cta_pairs else 1
+    cfg.options[TT_OPT_PLAIN_LAUNCHES] = 1 if plain_launches else 0
+    cfg.options[TT_OPT_FEED_FORWARD] = 0 if getattr(wl, "recurrent", True) else 1
+    cfg.options[TT_OPT_CTA_PAIRS] = 1 if cta_pairs else 0
+    cfg.options[TT_OPT_NO_POST_TC] = 0 if post_tc else 1
+    cfg.options[TT_OPT_RESERVED_SMS] = reserved_sms
     return cfg
 
 
@@ -207,7 +213,8 @@ class Context:
         for l in range(cfg.n_enc):
             w.enc_w[l] = ptr(weights[f"enc_w{l}"]).value
             w.enc_b[l] = ptr(weights[f"enc_b{l}"]).value
-        w.lstm_w, w.lstm_b = ptr(weights["lstm_w"]), ptr(weights["lstm_b"])
+        if "lstm_w" in weights:
+            w.lstm_w, w.lstm_b = ptr(weights["lstm_w"]), ptr(weights["lstm_b"])
         w.head_w, w.head_b = ptr(weights["head_w"]), ptr(weights["head_b"])
         if "conf_w" in weights:
             w.conf_w, w.conf_b = ptr(weights["conf_w"]), ptr(weights["conf_b"])
@@ -545,5 +552,19 @@ def overlay(src, src_w: int, src_h: int, src_pitch: int, masks, palette, stream=
     dst = torch.empty((K, src_h, src_w, 4), dtype=torch.uint8, device=src.device)
     st = lib.tt_overlay(src.data_ptr(), K, src.stride(0), src_w, src_h, src_pitch, masks.data_ptr(), T, hm, wm,
                         pal.ctypes.data, dst.data_ptr(), _stream_ptr(stream))
+    _check(lib, st, None)
+    return dst
+
+
+def render_layers(src, src_w: int, src_h: int, src_pitch: int, masks, palette, layers: int, carve_ctas: int = 0, stream=None,
+                  out=None):
+    """tt_render_layers: src uint8 CUDA [K][src_h*src_pitch], masks uint8 CUDA [K][T][Hm][Wm] -> uint8 [K][src_h][src_w][4]."""
+    import torch
+    lib = load_library()
+    K, T, hm, wm = masks.shape
+    pal = np.ascontiguousarray(np.asarray(palette, np.uint8)[:T]).reshape(-1)
+    dst = out if out is not None else torch.empty((K, src_h, src_w, 4), dtype=torch.uint8, device=src.device)
+    st = lib.tt_render_layers(src.data_ptr(), K, src.stride(0), src_w, src_h, src_pitch, masks.data_ptr(), T, hm, wm,
+                              pal.ctypes.data, layers, carve_ctas, dst.data_ptr(), _stream_ptr(stream))
     _check(lib, st, None)
     return dst

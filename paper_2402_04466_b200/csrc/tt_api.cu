@@ -108,6 +108,8 @@ struct tt_ctx {
   float *head_w = nullptr, *head_b = nullptr, *conf_w = nullptr, *conf_b = nullptr;
   float zthr = 0.f;
 
+  PostTcParams post_tc{};       // bf16 path: mask and confidence heads on the tensor cores when the hidden width allows
+  bool use_post_tc = false;
   ConvFirstTcParams first_tc{}; // bf16 path, first encoder layer on the tensor cores when its width (32 or 64) allows
   bool use_first_tc = false;
   SimtLayer simt_enc[TT_MAX_ENC];
@@ -148,7 +150,8 @@ struct tt_ctx {
   };
   std::vector<TickGraph> graphs;
   bool graphs_off = false;
-  bool no_pairs = false;            // reserved_[2]: never run the tensor-core layers on CTA pairs
+  bool cta_pairs = false;           // TT_OPT_CTA_PAIRS
+  bool feed_forward = false;        // TT_OPT_FEED_FORWARD: no recurrent cell, the heads read the encoder output
   const uint8_t** frame_tab_dev[2] = {nullptr, nullptr};   // device, [TT_MAX_STREAMS] pointers per slot
   const uint8_t** frame_tab_host[2] = {nullptr, nullptr};  // pinned staging of the same
   const uint8_t* const* cur_tab = nullptr;                  // table the tick being enqueued reads
@@ -402,7 +405,10 @@ tt_status validate(const tt_config* c, const tt_weights* w) {
   if (c->precision != TT_FP32 && c->precision != TT_BF16) return fail(nullptr, TT_ERR_INVALID_ARG, "bad precision");
   if (c->conf_mode != TT_CONF_MEAN_SIGMOID && c->conf_mode != TT_CONF_GAP_LINEAR) return fail(nullptr, TT_ERR_INVALID_ARG, "bad conf_mode");
   if (!(c->threshold > 0.f && c->threshold < 1.f)) return fail(nullptr, TT_ERR_INVALID_ARG, "threshold must lie in (0,1)");
-  if (!w->lstm_w || !w->lstm_b || !w->head_w || !w->head_b) return fail(nullptr, TT_ERR_INVALID_ARG, "missing weights");
+  const bool ff = c->options[TT_OPT_FEED_FORWARD] != 0;
+  if ((!ff && (!w->lstm_w || !w->lstm_b)) || !w->head_w || !w->head_b) return fail(nullptr, TT_ERR_INVALID_ARG, "missing weights");
+  if (ff && c->hidden != c->enc_cout[c->n_enc - 1])
+    return fail(nullptr, TT_ERR_INVALID_ARG, "a feed-forward model's `hidden` must equal its last encoder width (the heads read the encoder output)");
   if (c->conf_mode == TT_CONF_GAP_LINEAR && (!w->conf_w || !w->conf_b)) return fail(nullptr, TT_ERR_INVALID_ARG, "missing confidence-head weights");
   return TT_OK;
 }
@@ -413,6 +419,12 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
   TT_CUDA(ctx, cudaGetDeviceProperties(&prop, ctx->dev));
   if (prop.major != 10) return fail(ctx, TT_ERR_UNSUPPORTED, "device %d is sm_%d%d; this library is built for sm_100a only", ctx->dev, prop.major, prop.minor);
   ctx->sm_count = prop.multiProcessorCount;
+  // multiprocessors left to another workload (TT_OPT_RESERVED_SMS): the persistent kernels size their grids for the rest
+  if (c.options[TT_OPT_RESERVED_SMS] != 0) {
+    if ((int)c.options[TT_OPT_RESERVED_SMS] > ctx->sm_count / 2)
+      return fail(ctx, TT_ERR_INVALID_ARG, "at most half of the device's %d multiprocessors can be reserved", ctx->sm_count);
+    ctx->sm_count -= (int)c.options[TT_OPT_RESERVED_SMS];
+  }
   if (c.cuda_stream) {
     ctx->stream = reinterpret_cast<cudaStream_t>(c.cuda_stream);
   } else {
@@ -497,8 +509,10 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
     for (int k = 0; k <= TT_STAGE_COUNT; ++k) TT_CUDA(ctx, cudaEventCreate(&sl.stage_ev[k]));
   }
   bind_slot(ctx, 0);
-  ctx->graphs_off = c.reserved_[0] != 0;
-  ctx->no_pairs = c.reserved_[2] != 0;
+  ctx->graphs_off = c.options[TT_OPT_PLAIN_LAUNCHES] != 0;
+  ctx->cta_pairs = c.options[TT_OPT_CTA_PAIRS] != 0;
+  ctx->feed_forward = c.options[TT_OPT_FEED_FORWARD] != 0;
+  const bool no_post_tc = c.options[TT_OPT_NO_POST_TC] != 0;
 
   // ---- weights
   const bool r = ctx->bf16;  // round weights to bf16 on the bf16 path
@@ -519,7 +533,8 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
       if ((st = pack_simt(ctx, &ctx->simt_enc[l], w->enc_w[l], w->enc_b[l], ctx->lay_c[l], ctx->lay_c[l + 1],
                           c.enc_stride[l], ctx->lay_c[l + 1] > 16 ? 32 : 16, 0, false)) != TT_OK)
         return st;
-    if ((st = pack_simt(ctx, &ctx->simt_lstm, w->lstm_w, w->lstm_b, ctx->Cx + ctx->Ch, 4 * ctx->Ch, 1,
+    if (!ctx->feed_forward &&
+        (st = pack_simt(ctx, &ctx->simt_lstm, w->lstm_w, w->lstm_b, ctx->Cx + ctx->Ch, 4 * ctx->Ch, 1,
                         ctx->Ch >= 8 ? 32 : 16, ctx->Ch, false)) != TT_OK)
       return st;
   } else {
@@ -565,11 +580,46 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
         return st;
     }
     TcLayer& L = ctx->tc_lstm;
-    if ((st = pack_tc(ctx, &L, w->lstm_w, w->lstm_b, ctx->Cx, ctx->Ch, 4 * ctx->Ch, 1, ctx->Ch)) != TT_OK) return st;
-    if ((st = make_act_maps(ctx, &L.maps_a[0], reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[c.n_enc - 1]), S, ctx->Hm,
-                            ctx->Wm, ctx->Cx, 1, L.slab_c)) != TT_OK)
-      return st;
-    if ((st = make_act_maps(ctx, &L.maps_a[4], ctx->h_bf16, 2 * S, ctx->Hm, ctx->Wm, ctx->Ch, 1, L.slab_c)) != TT_OK) return st;
+    if (!ctx->feed_forward) {
+      if ((st = pack_tc(ctx, &L, w->lstm_w, w->lstm_b, ctx->Cx, ctx->Ch, 4 * ctx->Ch, 1, ctx->Ch)) != TT_OK) return st;
+      if ((st = make_act_maps(ctx, &L.maps_a[0], reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[c.n_enc - 1]), S, ctx->Hm,
+                              ctx->Wm, ctx->Cx, 1, L.slab_c)) != TT_OK)
+        return st;
+      if ((st = make_act_maps(ctx, &L.maps_a[4], ctx->h_bf16, 2 * S, ctx->Hm, ctx->Wm, ctx->Ch, 1, L.slab_c)) != TT_OK) return st;
+    } else if (no_post_tc || !post_tc_supported(ctx->Ch, (int)plane)) {
+      return fail(ctx, TT_ERR_UNSUPPORTED, "a bf16 feed-forward model needs a last encoder width in multiples of 64 (at most 512) and "
+                                           "a map of at least 128 pixels: its heads run on the tensor cores only");
+    }
+    if (!no_post_tc && post_tc_supported(ctx->Ch, (int)plane)) {
+      // packed weights of both heads, bf16 [16][Ch] (the context's head weights are bf16 values already)
+      std::vector<uint16_t> pw((size_t)16 * ctx->Ch, 0);
+      for (int t = 0; t < ctx->T; ++t)
+        for (int ch = 0; ch < ctx->Ch; ++ch) {
+          pw[(size_t)t * ctx->Ch + ch] = f32_to_bf16_rne(w->head_w[(size_t)t * ctx->Ch + ch]);
+          if (c.conf_mode == TT_CONF_GAP_LINEAR) pw[(size_t)(8 + t) * ctx->Ch + ch] = f32_to_bf16_rne(w->conf_w[(size_t)t * ctx->Ch + ch]);
+        }
+      uint16_t* dpw = nullptr;
+      if ((st = upload(ctx, &dpw, pw)) != TT_OK) return st;
+      PostTcParams& q = ctx->post_tc;
+      {
+        // the heads' input: the bf16 copy of the new hidden state, or a feed-forward model's last encoder output
+        const cuuint64_t dims[3] = {(cuuint64_t)ctx->Ch, (cuuint64_t)plane, (cuuint64_t)(ctx->feed_forward ? S : 2 * S)};
+        const cuuint64_t str[2] = {(cuuint64_t)ctx->Ch * 2, (cuuint64_t)plane * ctx->Ch * 2};
+        const cuuint32_t box[3] = {64, 128, 1};
+        void* src = ctx->feed_forward ? ctx->enc_out[c.n_enc - 1] : static_cast<void*>(ctx->h_bf16);
+        if ((st = encode_map(ctx, &q.map_h, src, 3, dims, str, box, 128)) != TT_OK) return st;
+      }
+      {
+        const cuuint64_t dims[2] = {(cuuint64_t)ctx->Ch, 16};
+        const cuuint64_t str[1] = {(cuuint64_t)ctx->Ch * 2};
+        const cuuint32_t box[2] = {64, 16};
+        if ((st = encode_map(ctx, &q.map_w, dpw, 2, dims, str, box, 128)) != TT_OK) return st;
+      }
+      q.Hm = ctx->Hm; q.Wm = ctx->Wm; q.T = ctx->T; q.kslabs = ctx->Ch / 64;
+      q.head_b = ctx->head_b; q.conf_b = ctx->conf_b; q.conf_mode = c.conf_mode; q.zthr = ctx->zthr;
+      q.scratch = ctx->post_scratch; q.status = ctx->status_dev; q.wait_limit = ctx->wait_limit;
+      ctx->use_post_tc = true;
+    }
   }
   for (int i = 0; i < TT_MAX_STREAMS; ++i) {
     ctx->states[i].ctx = ctx;
@@ -656,6 +706,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
       if ((ms_ = mark_stage(ctx, TT_STAGE_ENC0 + l, 1)) != TT_OK) return ms_;
       in = reinterpret_cast<const float*>(ctx->enc_out[l]);
     }
+    if (!ctx->feed_forward) {
     const SimtLayer& L = ctx->simt_lstm;
     ConvSimtParams q{};
     q.in0 = in; q.img_stride0 = (int64_t)ctx->Cx * plane; q.idx0 = ident; q.C0 = ctx->Cx;
@@ -666,6 +717,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
     q.hidden = ctx->Ch;
     TT_CUDA(ctx, launch_conv_simt(q, s));
     if ((ms_ = mark_stage(ctx, TT_STAGE_CONVLSTM, 1)) != TT_OK) return ms_;
+    }
   } else {
     if (ctx->use_first_tc) {
       ctx->first_tc.K = K;
@@ -691,8 +743,8 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
       if (bi < 0) return fail(ctx, TT_ERR_UNSUPPORTED, "no tensor-core tile shape fits this layer");
       const int bns[3] = {64, 128, 256};
       q.block_n = bns[bi]; q.map_b = L.map_b[bi]; q.n_tiles_n = L.cout / q.block_n;
-      // 256-wide tiles run on CTA pairs: each CTA stages its own activation box and half of the weight slab
-      q.pair = (bi == 2 && L.slab_c == 64 && L.has_b[1] && !ctx->no_pairs && K * q.tiles_x * q.tiles_y >= 2) ? 1 : 0;
+      // on request 256-wide tiles run on CTA pairs: each CTA stages its own activation box and half of the weight slab
+      q.pair = (bi == 2 && L.slab_c == 64 && L.has_b[1] && ctx->cta_pairs && K * q.tiles_x * q.tiles_y >= 2) ? 1 : 0;
       if (q.pair) q.map_b = L.map_b[1];
       q.cout = L.cout; q.bias = L.b; q.status = ctx->status_dev; q.wait_limit = ctx->wait_limit;
       q.n_prod = 3;
@@ -709,6 +761,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
       TT_CUDA(ctx, launch_conv_tc(q, ctx->sm_count, s));
       if ((ms_ = mark_stage(ctx, TT_STAGE_ENC0 + l, 1)) != TT_OK) return ms_;
     }
+    if (!ctx->feed_forward) {
     const TcLayer& L = ctx->tc_lstm;
     ConvTcParams q{};
     tt_status st = fill_common(q, L, ctx->Hm, ctx->Wm);
@@ -718,11 +771,24 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
     q.c_idx = c_idx; q.h_out_idx = h_out; q.hidden = ctx->Ch;
     TT_CUDA(ctx, launch_conv_tc(q, ctx->sm_count, s));
     if ((ms_ = mark_stage(ctx, TT_STAGE_CONVLSTM, 1)) != TT_OK) return ms_;
+    }
   }
 
+  if (ctx->use_post_tc) {
+    PostTcParams& q = ctx->post_tc;
+    q.idx = ctx->feed_forward ? ident : h_out; q.K = K;
+    q.logits = ctx->logits; q.probs = ctx->probs; q.masks = ctx->masks; q.bits = ctx->bits; q.results = ctx->results_dev;
+    q.pdl = ctx->profiling ? 0 : 1;
+    TT_CUDA(ctx, launch_post_tc(q, ctx->sm_count, s));
+    if ((ms_ = mark_stage(ctx, TT_STAGE_POSTPROCESS, 1)) != TT_OK) return ms_;
+  } else {
   PostParams po{};
   po.h = ctx->h_f32; po.channels_last = ctx->bf16 ? 1 : 0; po.img_stride = (int64_t)ctx->Ch * plane;
   po.idx = ctx->bf16 ? c_idx : h_out;
+  if (ctx->feed_forward) {   // fp32 path: the heads read the planar output of the last encoder layer
+    po.h = reinterpret_cast<const float*>(ctx->enc_out[ctx->n_enc - 1]);
+    po.idx = ident;
+  }
   po.K = K; po.Hm = ctx->Hm; po.Wm = ctx->Wm; po.Ch = ctx->Ch; po.T = ctx->T;
   po.head_w = ctx->head_w; po.head_b = ctx->head_b; po.conf_w = ctx->conf_w; po.conf_b = ctx->conf_b;
   po.conf_mode = c.conf_mode; po.zthr = ctx->zthr;
@@ -730,7 +796,8 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
   po.results = ctx->results_dev; po.scratch = ctx->post_scratch; po.status = ctx->status_dev; po.wait_limit = ctx->wait_limit;
   po.pdl = (ctx->bf16 && !ctx->profiling) ? 1 : 0;
   TT_CUDA(ctx, launch_postprocess(po, s));
-  if ((ms_ = mark_stage(ctx, TT_STAGE_POSTPROCESS, 2)) != TT_OK) return ms_;
+  if ((ms_ = mark_stage(ctx, TT_STAGE_POSTPROCESS, 1)) != TT_OK) return ms_;
+  }
 
   if (c.overlay) {
     OverlayParams ov{};
@@ -835,6 +902,7 @@ tt_status tt_state_reset(tt_ctx* ctx, tt_state* st) {
 tt_status tt_state_export(tt_ctx* ctx, tt_state* st, float* h_host, float* c_host) {
   if (!ctx || !owns_state(ctx, st) || !h_host || !c_host) return ctx ? fail(ctx, TT_ERR_INVALID_ARG, "bad state or null buffer") : TT_ERR_INVALID_ARG;
   if (ctx->q_count) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
+  if (ctx->feed_forward) return fail(ctx, TT_ERR_UNSUPPORTED, "a feed-forward model has no recurrent state");
   TT_CUDA(ctx, cudaSetDevice(ctx->dev));
   const int plane = ctx->Hm * ctx->Wm;
   const size_t n = (size_t)ctx->Ch * plane;
@@ -855,6 +923,7 @@ tt_status tt_state_export(tt_ctx* ctx, tt_state* st, float* h_host, float* c_hos
 tt_status tt_state_import(tt_ctx* ctx, tt_state* st, const float* h_host, const float* c_host) {
   if (!ctx || !owns_state(ctx, st) || !h_host || !c_host) return ctx ? fail(ctx, TT_ERR_INVALID_ARG, "bad state or null buffer") : TT_ERR_INVALID_ARG;
   if (ctx->q_count) return fail(ctx, TT_ERR_NOT_READY, "a submit is in flight");
+  if (ctx->feed_forward) return fail(ctx, TT_ERR_UNSUPPORTED, "a feed-forward model has no recurrent state");
   TT_CUDA(ctx, cudaSetDevice(ctx->dev));
   const int plane = ctx->Hm * ctx->Wm;
   const size_t n = (size_t)ctx->Ch * plane;
@@ -1274,6 +1343,25 @@ tt_status tt_overlay(const uint8_t* src_dev, int32_t K, int64_t src_frame_stride
   p.dst = dst_dev;
   cudaError_t e = launch_overlay(p, reinterpret_cast<cudaStream_t>(cuda_stream));
   if (e != cudaSuccess) return fail(nullptr, TT_ERR_CUDA, "tt_overlay: %s", cudaGetErrorString(e));
+  return TT_OK;
+}
+
+tt_status tt_render_layers(const uint8_t* src_dev, int32_t K, int64_t src_frame_stride, int32_t src_w, int32_t src_h,
+                           int32_t src_pitch, const uint8_t* masks_dev, int32_t n_tools, int32_t hm, int32_t wm,
+                           const uint8_t* palette_host, int32_t layers, int32_t carve_ctas, uint8_t* dst_dev,
+                           void* cuda_stream) {
+  if (!src_dev || !masks_dev || !palette_host || !dst_dev || K < 1 || K > TT_MAX_STREAMS || src_w < 1 || src_h < 1 ||
+      src_w > 16384 || src_h > 16384 || src_pitch < 3 * src_w || n_tools < 1 || n_tools > TT_MAX_TOOLS || hm < 1 || wm < 1 ||
+      hm > 16384 || wm > 16384 || layers < 1 || layers > 4096 || carve_ctas < 0 || carve_ctas > 65535)
+    return fail(nullptr, TT_ERR_INVALID_ARG, "tt_render_layers: bad argument");
+  if (misaligned(dst_dev, 4)) return fail(nullptr, TT_ERR_INVALID_ARG, "tt_render_layers: dst_dev must be 4-byte aligned");
+  RenderParams p{};
+  for (int n = 0; n < K; ++n) p.src.p[n] = src_dev + (size_t)n * src_frame_stride;
+  p.K = K; p.src_w = src_w; p.src_h = src_h; p.src_pitch = src_pitch; p.T = n_tools; p.Hm = hm; p.Wm = wm;
+  p.masks = masks_dev; p.layers = layers; p.carve_ctas = carve_ctas; p.dst = dst_dev;
+  std::memcpy(p.palette, palette_host, (size_t)n_tools * 3);
+  cudaError_t e = launch_render(p, reinterpret_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return fail(nullptr, TT_ERR_CUDA, "tt_render_layers: %s", cudaGetErrorString(e));
   return TT_OK;
 }
 

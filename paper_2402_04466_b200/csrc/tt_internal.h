@@ -178,6 +178,29 @@ cudaError_t launch_postprocess(const PostParams& p, cudaStream_t s);
 cudaError_t post_prepare();
 cudaError_t post_static_scratch(void** ptr);  // device address of the library's built-in scratch array
 
+// S4/S5 of the bf16 path on the tensor cores: reads the bf16 channels-last hidden state.
+struct PostTcParams {
+  TensorMap128 map_h;     // bf16 [n_img][plane][Ch], box [64 channels][128 pixels][1], 128-byte swizzle
+  TensorMap128 map_w;     // bf16 [16][Ch]: rows 0..7 head weights, rows 8..15 confidence-head weights; box [64][16]
+  IdxMap idx;             // image index of batch position n inside the hidden-state tensor
+  int32_t K, Hm, Wm, T, kslabs;   // kslabs = Ch / 64
+  const float* head_b;
+  const float* conf_b;    // null for TT_CONF_MEAN_SIGMOID
+  int32_t conf_mode;
+  float zthr;
+  float* logits;          // [K][T][plane]
+  float* probs;
+  uint8_t* masks;
+  uint8_t* bits;          // optional [K][plane]
+  tt_result* results;     // device, [K]
+  void* scratch;          // post_scratch_bytes(...) bytes, zero on entry, zero again on exit
+  int32_t* status;
+  long long wait_limit;
+  int32_t pdl;
+};
+bool post_tc_supported(int ch, int plane);
+cudaError_t launch_post_tc(const PostTcParams& p, int sm_count, cudaStream_t s);
+
 // -------------------------------------------------------------------------- S6 overlay
 struct OverlayParams {
   FramePtrs src;
@@ -189,6 +212,18 @@ struct OverlayParams {
   uint8_t* dst;          // [K][src_h][src_w][4]
 };
 cudaError_t launch_overlay(const OverlayParams& p, cudaStream_t s);
+
+// ------------------------------------------- scaled-up visualisation load (multi-layer blend)
+struct RenderParams {
+  FramePtrs src;
+  int32_t K, src_w, src_h, src_pitch, T, Hm, Wm;
+  const uint8_t* masks;   // [K][T][plane]
+  uint8_t palette[TT_MAX_TOOLS][3];
+  int32_t layers;         // the S6 blend is applied this many times, layer l with the palette rotated by l
+  int32_t carve_ctas;     // 0: one block per 1024 pixels over the whole device; > 0: that many looping blocks
+  uint8_t* dst;           // [K][src_h][src_w][4]
+};
+cudaError_t launch_render(const RenderParams& p, cudaStream_t s);
 
 // ------------------------------------------------------------------------ layout helpers
 // fp32 NCHW <-> internal layouts, used by state import/export and debug taps.

@@ -13,7 +13,7 @@ from parity_util import assert_close, check_masks, check_reductions_from_own_mas
 pytestmark = pytest.mark.gpu
 
 
-def _make(wl, K=1, overlay=None, precision=None, timeout_ns=0, plain_launches=False, cta_pairs=True):
+def _make(wl, K=1, overlay=None, precision=None, timeout_ns=0, plain_launches=False, cta_pairs=False):
     weights = tt_synth.make_weights(wl)
     cfg = binding.make_config(wl, max_streams=K, overlay=overlay, precision=precision, sync_timeout_ns=timeout_ns,
                               plain_launches=plain_launches, cta_pairs=cta_pairs)
@@ -46,8 +46,9 @@ def _compare_frame(ctx, st, res, ref, tol, band, check_tensors=True, tag="", tol
         stats["pre"] = assert_close(ctx.debug_tensor(st, "pre"), ref.pre, 1e-4, tag + " pre")
         for l, e in enumerate(ref.enc):
             stats[f"enc{l}"] = assert_close(ctx.debug_tensor(st, f"enc{l}"), e, tol_mid, tag + f" enc{l}")
-        stats["c"] = assert_close(ctx.debug_tensor(st, "c"), ref.c, tol_mid, tag + " c")
-        stats["h"] = assert_close(ctx.debug_tensor(st, "h"), ref.h, tol_mid, tag + " h")
+        if not ctx.cfg.options[binding.TT_OPT_FEED_FORWARD]:          # a feed-forward model carries no state
+            stats["c"] = assert_close(ctx.debug_tensor(st, "c"), ref.c, tol_mid, tag + " c")
+            stats["h"] = assert_close(ctx.debug_tensor(st, "h"), ref.h, tol_mid, tag + " h")
         stats["logits"] = assert_close(ctx.debug_tensor(st, "logits"), ref.z, tol_mid, tag + " logits")
     stats["prob"] = assert_close(ctx.fetch_probs(res), ref.p, tol, tag + " prob")
     stats["conf"] = assert_close(res["conf"], ref.conf, tol, tag + " conf")
@@ -139,8 +140,8 @@ TOL_OUT, TOL_MID_PLAIN, TOL_MIRROR, TOL_MIRROR_RMS = 2e-2, 5e-2, 2e-2, 3e-3
 BAND_REL, MAX_BAND_FRAC = 2e-2, 0.05
 
 
-def _run_bf16(cuda_device, wl, K, n_frames, tol_plain=TOL_OUT, tol_mirror=TOL_MIRROR, overlay=False):
-    ctx, states, w = _make(wl, K, overlay=overlay)
+def _run_bf16(cuda_device, wl, K, n_frames, tol_plain=TOL_OUT, tol_mirror=TOL_MIRROR, overlay=False, cta_pairs=False):
+    ctx, states, w = _make(wl, K, overlay=overlay, cta_pairs=cta_pairs)
     plain = [oracle.OraclePipeline(wl, w) for _ in range(K)]
     mirror = [oracle.OraclePipeline(wl, w, mirror_bf16=True) for _ in range(K)]
     frames = _frames(wl, K, n_frames)
@@ -225,12 +226,12 @@ def test_bf16_wide_channels_small_map(cuda_device):
 
 
 def test_bf16_cta_pairs_with_an_odd_number_of_tiles(cuda_device):
-    """The 256-wide ConvLSTM tiles run on CTA pairs (two neighbouring 128-pixel tiles per MMA).  Three streams of
-    an 80x40 map give 75 tiles: the last pair has no second tile, its second CTA recomputes the last tile and
-    must store nothing.  Checked against the oracle, and bit for bit against the same context without pairs."""
+    """On request the 256-wide ConvLSTM tiles run on CTA pairs (two neighbouring 128-pixel tiles per MMA).  Three
+    streams of an 80x40 map give 75 tiles: the last pair has no second tile, its second CTA recomputes the last
+    tile and must store nothing.  Checked against the oracle, and bit for bit against the default single-CTA tiles."""
     wl = tt_synth.workload("cfg1-gain").with_(name="bf16-pairs", src_w=854, src_h=320, net_w=640, net_h=320)
     assert wl.map_hw() == (40, 80)
-    _run_bf16(cuda_device, wl, 3, 2)
+    _run_bf16(cuda_device, wl, 3, 2, cta_pairs=True)
     K, n = 3, 2
     frames = _frames(wl, K, n)
     outs = []
@@ -244,6 +245,37 @@ def test_bf16_cta_pairs_with_an_odd_number_of_tiles(cuda_device):
     for k in range(K):
         assert np.array_equal(outs[0][0][k][0], outs[1][0][k][0]) and np.array_equal(outs[0][0][k][1], outs[1][0][k][1])
         assert np.array_equal(outs[0][1][k], outs[1][1][k])
+
+
+def test_bf16_postprocess_from_the_fp32_state_still_matches(cuda_device):
+    """By default the bf16 path forms the mask and confidence heads on the tensor cores from the bf16 copy of the
+    hidden state (every other bf16 test runs that way).  The kernel that reads the fp32 state instead stays
+    available; both must match the oracle, and each other within twice the output tolerance."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="post-fp32", src_w=214, src_h=120, net_w=160, net_h=120)
+    K, n = 2, 2
+    frames = _frames(wl, K, n)
+    w = tt_synth.make_weights(wl)
+    ctxs = []
+    for post_tc in (True, False):
+        ctx = binding.Context(binding.make_config(wl, max_streams=K, post_tc=post_tc), w)
+        ctxs.append((ctx, [ctx.state_create() for _ in range(K)]))
+    oras = [oracle.OraclePipeline(wl, w) for _ in range(K)]
+    for t in range(n):
+        refs = [oras[k].step(frames[k][t], want_overlay=False) for k in range(K)]
+        got = []
+        for ctx, states in ctxs:
+            ctx.submit_frames([torch.from_numpy(frames[k][t]).to(cuda_device) for k in range(K)], states, frame_index=t)
+            res = ctx.sync()
+            for k in range(K):
+                band = max(1e-3, BAND_REL * float(np.sqrt(np.mean(refs[k].z.astype(np.float64) ** 2))))
+                _compare_frame(ctx, states[k], res[k], refs[k], TOL_OUT, band, tag=f"post-fp32 k={k} t={t}", tol_mid=TOL_MID_PLAIN,
+                               max_band_frac=MAX_BAND_FRAC)
+            got.append([(ctx.fetch_probs(r), r["conf"].copy()) for r in res])
+        for k in range(K):
+            assert_close(got[0][k][0], got[1][k][0], 2 * TOL_OUT, "probabilities of the two postprocess kernels")
+            assert_close(got[0][k][1], got[1][k][1], 2 * TOL_OUT, "confidences of the two postprocess kernels")
+    for ctx, _ in ctxs:
+        ctx.destroy()
 
 
 def test_bf16_stride1_encoder_and_overlay(cuda_device):
@@ -506,6 +538,77 @@ def test_boundary_error_paths(cuda_device):
     with pytest.raises(binding.TTError) as e:
         binding.Context(binding.make_config(bad), tt_synth.make_weights(bad))
     assert e.value.status == 2
+
+
+def test_feed_forward_model_bf16_and_fp32(cuda_device):
+    """The second workload class of the paper (Section V-B: a feed-forward segmentation network): the same encoder
+    and heads without the recurrent cell.  Both precision paths against the oracle; results must not depend on
+    earlier frames; state calls are refused."""
+    for wl, K, tol, band_rel, tol_mid in (
+            (tt_synth.workload("cfg1-ff-gain").with_(name="ff-bf16", src_w=214, src_h=120, net_w=176, net_h=136), 3, TOL_OUT, BAND_REL, TOL_MID_PLAIN),
+            (tt_synth.workload("cfg0-ff-gain").with_(name="ff-fp32", src_w=150, src_h=110, net_w=100, net_h=76, enc_cout=(8, 24), enc_stride=(2, 2),
+                                                     hidden=24, n_tools=5, conf_mode="gap_linear", frame_kind="endoscopy"), 2, 1e-4, 0.0, 1e-4)):
+        ctx, states, w = _make(wl, K)
+        assert "lstm_w" not in w
+        oras = [oracle.OraclePipeline(wl, w) for _ in range(K)]
+        frames = _frames(wl, K, 3)
+        first = None
+        for t in (0, 1, 2, 0):                                        # frame 0 again at the end: same result as the first time
+            ctx.submit_frames([torch.from_numpy(frames[k][t]).to(cuda_device) for k in range(K)], states, frame_index=t)
+            res = ctx.sync()
+            for k in range(K):
+                ref = oras[k].step(frames[k][t], want_overlay=False)
+                band = max(1e-3, band_rel * float(np.sqrt(np.mean(ref.z.astype(np.float64) ** 2))))
+                _compare_frame(ctx, states[k], res[k], ref, tol, band, tag=f"{wl.name} k={k} t={t}", tol_mid=tol_mid)
+            snap = [(ctx.fetch_probs(r), r["conf"].copy(), r["count"].copy()) for r in res]
+            if first is None:
+                first = snap
+        for a, b in zip(first, snap):
+            assert all(np.array_equal(x, y) for x, y in zip(a, b))
+        with pytest.raises(binding.TTError) as e:
+            ctx.state_export(states[0])
+        assert e.value.status == 2
+        ctx.destroy()
+    # hidden must be the last encoder width
+    bad = tt_synth.workload("cfg1-ff").with_(hidden=64)
+    with pytest.raises(binding.TTError) as e:
+        binding.Context(binding.make_config(bad), tt_synth.make_weights(bad.with_(hidden=128)))
+    assert e.value.status == 1
+
+
+def test_two_models_in_the_same_tick_match_their_solo_runs(cuda_device):
+    """Heterogeneous concurrency (the paper's Section VI experiment with two different applications on one GPU): a
+    recurrent tool-tracking model and a feed-forward segmentation model, each a context with its own CUDA stream,
+    are submitted in the same tick and run concurrently.  Each must return bit for bit what it returns alone."""
+    wa = tt_synth.workload("cfg1-gain").with_(name="het-rec", src_w=214, src_h=120, net_w=160, net_h=120)
+    wb = tt_synth.workload("cfg1-ff-gain").with_(name="het-ff", src_w=320, src_h=200, net_w=256, net_h=160, enc_cout=(32, 64, 64), hidden=64)
+    n = 4
+    fa, fb = _frames(wa, 2, n), _frames(wb, 3, n)
+
+    def collect(ctx, res):
+        return [(ctx.fetch_probs(r), r["conf"].copy(), r["count"].copy(), r["cx"].copy()) for r in res]
+
+    solo = {}
+    for name, wl, K, frames in (("a", wa, 2, fa), ("b", wb, 3, fb)):
+        ctx, states, _ = _make(wl, K)
+        solo[name] = []
+        for t in range(n):
+            ctx.submit_frames([torch.from_numpy(frames[k][t]).to(cuda_device) for k in range(K)], states, frame_index=t)
+            solo[name].append(collect(ctx, ctx.sync()))
+        ctx.destroy()
+    (ca, sa, _), (cb, sb, w_b) = _make(wa, 2), _make(wb, 3)
+    ora_b = oracle.OraclePipeline(wb, w_b)
+    for t in range(n):
+        ca.submit_frames([torch.from_numpy(fa[k][t]).to(cuda_device) for k in range(2)], sa, frame_index=t)
+        cb.submit_frames([torch.from_numpy(fb[k][t]).to(cuda_device) for k in range(3)], sb, frame_index=t)   # both in flight
+        ra, rb = ca.sync(), cb.sync()
+        for got, want in ((collect(ca, ra), solo["a"][t]), (collect(cb, rb), solo["b"][t])):
+            for g, w_ in zip(got, want):
+                assert all(np.array_equal(x, y) for x, y in zip(g, w_))
+        ref = ora_b.step(fb[0][t], want_overlay=False)
+        assert_close(cb.fetch_probs(rb[0]), ref.p, TOL_OUT, f"feed-forward model in a shared tick t={t}")
+    ca.destroy()
+    cb.destroy()
 
 
 def test_host_side_sync_timeout_leaves_the_submit_in_flight(cuda_device):

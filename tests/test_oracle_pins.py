@@ -312,3 +312,62 @@ def test_oracle_bf16_rounding_spread():
     mid = max(rel_err(b.enc[1], a.enc[1]), rel_err(b.h, a.h), rel_err(b.c, a.c))
     assert 1e-2 < mid < 5e-2
     assert rel_err(b.p, a.p) < 1e-2
+
+
+def test_feed_forward_pipeline_is_the_composition_of_the_pinned_stages_and_stateless():
+    """The feed-forward variant (no recurrent cell) must be exactly encoder -> heads: composed here from torch
+    conv2d in fp64 and the textbook head formulas, and independent of whatever frames came before."""
+    import torch
+    import torch.nn.functional as F
+
+    import tt_synth
+    from oracle import OraclePipeline
+    wl = tt_synth.workload("cfg0-ff-gain").with_(src_w=40, src_h=32, net_w=24, net_h=20, enc_cout=(6, 10), enc_stride=(2, 1),
+                                                 hidden=10, n_tools=3, conf_mode="gap_linear")
+    w = tt_synth.make_weights(wl)
+    assert "lstm_w" not in w and w["head_w"].shape == (3, 10)
+    frames = tt_synth.make_frames(wl.frame_kind, wl.stream_seed(0), 3, wl.src_w, wl.src_h)
+    ora = OraclePipeline(wl, w)
+    outs = [ora.step(frames[t], want_overlay=False) for t in (0, 1, 2)]
+    again = ora.step(frames[0], want_overlay=False)
+    assert np.array_equal(again.z, outs[0].z) and np.array_equal(again.conf, outs[0].conf)      # no state carried
+    x = torch.from_numpy(outs[2].pre.astype(np.float64))[None]
+    for l, s in enumerate(wl.enc_stride):
+        x = F.relu(F.conv2d(x, torch.from_numpy(w[f"enc_w{l}"].astype(np.float64)), torch.from_numpy(w[f"enc_b{l}"].astype(np.float64)),
+                            stride=s, padding=1))
+    feat = x[0].numpy()
+    z = np.einsum("tc,chw->thw", w["head_w"].astype(np.float64), feat) + w["head_b"].astype(np.float64)[:, None, None]
+    assert np.allclose(outs[2].z, z, rtol=1e-5, atol=1e-6)
+    conf = 1.0 / (1.0 + np.exp(-(w["conf_w"].astype(np.float64) @ feat.mean(axis=(1, 2)) + w["conf_b"])))
+    assert np.allclose(outs[2].conf, conf, rtol=1e-5, atol=1e-6)
+    assert np.array_equal(outs[2].mask, (outs[2].z > 0).astype(np.uint8))
+
+
+def test_render_layers_pins():
+    """The multi-layer render load: one layer is the overlay itself; empty masks leave the frame alone; a pixel
+    covered by one tool goes through the integer blend once per layer with that layer's colour (by hand)."""
+    import oracle
+    frame = np.full((4, 6, 3), 0, np.uint8)
+    frame[..., 0], frame[..., 1], frame[..., 2] = 10, 200, 77
+    pal = [(255, 0, 0), (0, 255, 0), (0, 0, 255)]
+    mask = np.zeros((3, 2, 3), np.uint8)
+    out = oracle.render_layers(frame, mask, pal, 5)
+    assert np.array_equal(out[..., :3], frame) and np.all(out[..., 3] == 255)
+    mask[1, 0, 0] = 1                                   # tool 1 covers source pixels x in [0,2), y in [0,2)
+    assert np.array_equal(oracle.render_layers(frame, mask, pal, 1), oracle.overlay(frame, mask, pal))
+    out = oracle.render_layers(frame, mask, pal, 3)
+    rgb = [10, 200, 77]
+    for l in range(3):
+        c = pal[(1 + l) % 3]                            # layer l paints tool 1 with colour (1 + l) mod 3
+        rgb = [(153 * v + 102 * c[k] + 127) // 255 for k, v in enumerate(rgb)]
+    assert list(out[0, 0, :3]) == rgb and list(out[1, 1, :3]) == rgb
+    assert list(out[0, 2, :3]) == [10, 200, 77] and list(out[3, 5, :3]) == [10, 200, 77]
+    # two tools on one pixel: ascending tool order inside a layer
+    mask[2, 0, 0] = 1
+    out = oracle.render_layers(frame, mask, pal, 2)
+    rgb = [10, 200, 77]
+    for l in range(2):
+        for t in (1, 2):
+            c = pal[(t + l) % 3]
+            rgb = [(153 * v + 102 * c[k] + 127) // 255 for k, v in enumerate(rgb)]
+    assert list(out[0, 0, :3]) == rgb

@@ -41,6 +41,7 @@ class Workload:
     norm_mean: float = 0.5
     norm_std: float = 0.25
     gain_corrected: bool = False
+    recurrent: bool = True    # False: feed-forward model, the heads read the last encoder output (hidden == enc_cout[-1])
     seed: int = BASE_SEED
     palette: Tuple[Tuple[int, int, int], ...] = field(default=PALETTE)
 
@@ -81,8 +82,16 @@ _CFG4 = Workload("cfg4", 1920, 1080, 1280, 720, (64, 128, 256), (2, 2, 2), 256, 
 WORKLOADS = {w.name: w for w in (_CFG0, _CFG1, _CFG2, _CFG3, _CFG4)}
 
 
+def feed_forward_variant(wl: Workload) -> Workload:
+    """The same encoder and heads without the recurrent cell (a feed-forward segmentation model)."""
+    return replace(wl, name=wl.name + "-ff", recurrent=False, hidden=wl.enc_cout[-1])
+
+
 def workload(name: str) -> Workload:
-    """Look up 'cfg0'..'cfg4'; a '-gain' suffix selects the gain-corrected parity variant."""
+    """Look up 'cfg0'..'cfg4'; a '-gain' suffix selects the gain-corrected parity variant, a '-ff' suffix
+    (before '-gain') the feed-forward variant."""
     if name.endswith("-gain"):
-        return WORKLOADS[name[:-5]].parity_variant()
+        return workload(name[:-5]).parity_variant()
+    if name.endswith("-ff"):
+        return feed_forward_variant(workload(name[:-3]))
     return WORKLOADS[name]

@@ -29,7 +29,7 @@ def round_to_bf16(x: np.ndarray) -> np.ndarray:
 
 
 def make_weights(wl: Workload) -> Dict[str, np.ndarray]:
-    """Returns enc_w{l}, enc_b{l}, lstm_w, lstm_b, head_w, head_b and (gap_linear) conf_w, conf_b."""
+    """Returns enc_w{l}, enc_b{l}, lstm_w, lstm_b (recurrent models), head_w, head_b and (gap_linear) conf_w, conf_b."""
     seed = wl.weight_seed()
     tid = [100]
 
@@ -52,18 +52,21 @@ def make_weights(wl: Workload) -> Dict[str, np.ndarray]:
             w = round_to_bf16(w)
         out[f"enc_w{l}"], out[f"enc_b{l}"] = w, b
         cin = cout
-    ch = wl.hidden
-    fan_in = 9 * (cin + ch)
-    sw = math.sqrt(1.0 / fan_in) if wl.gain_corrected else wl.weight_sigma
+    recurrent = getattr(wl, "recurrent", True)
+    ch = wl.hidden if recurrent else cin
     sb = 0.05 if wl.gain_corrected else wl.weight_sigma
-    w = draw((4 * ch, cin + ch, 3, 3), sw)
-    b = draw((4 * ch,), sb)
-    if bf16:
-        w = round_to_bf16(w)
-    out["lstm_w"], out["lstm_b"] = w, b
+    if recurrent:
+        fan_in = 9 * (cin + ch)
+        sw = math.sqrt(1.0 / fan_in) if wl.gain_corrected else wl.weight_sigma
+        w = draw((4 * ch, cin + ch, 3, 3), sw)
+        b = draw((4 * ch,), sb)
+        if bf16:
+            w = round_to_bf16(w)
+        out["lstm_w"], out["lstm_b"] = w, b
     # Hidden activations are o*tanh(c') with rms around 0.1-0.3; scale the mask head so
-    # logits spread over a few units in the parity variant.
-    sw = 8.0 * math.sqrt(1.0 / ch) if wl.gain_corrected else wl.weight_sigma
+    # logits spread over a few units in the parity variant.  A feed-forward model's heads read
+    # ReLU features of O(1) size instead.
+    sw = (8.0 if recurrent else 1.0) * math.sqrt(1.0 / ch) if wl.gain_corrected else wl.weight_sigma
     out["head_w"] = draw((wl.n_tools, ch), sw)
     if bf16:
         out["head_w"] = round_to_bf16(out["head_w"])
