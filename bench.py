@@ -341,6 +341,200 @@ def staggered_run(ctx, states, host_ring, K, R, n_frames, window_ns, seed):
     return out
 
 
+# ------------------------------------------------- studies beyond the headline (run on request)
+def paced_multi(parts, n_frames, before_tick=None):
+    """Several contexts driven in lock step: every 16.667 ms the frames of all parts arrive together, every part is
+    submitted (each on its own context), then every part is synced in turn.  parts: list of dicts with ctx, states,
+    host_ring (pinned), K, R.  Returns per part the latency summary (arrival -> that part's tt_sync returned) and,
+    under "all", arrival -> the last part returned.  before_tick(i) runs right after the arrival of frame i."""
+    import ctypes as C
+
+    from paper_2402_04466_b200 import binding
+    from paper_2402_04466_b200.stats import latency_summary, trim_warmup
+    try:
+        os.sched_setaffinity(0, {sorted(os.sched_getaffinity(0))[-1]})
+    except Exception:
+        pass
+    for p in parts:
+        p["fr"] = (binding.tt_frame * p["K"])()
+        p["sts"] = (C.c_void_p * p["K"])(*[s.value for s in p["states"]])
+        p["res"] = (binding.tt_result * binding.TT_MAX_STREAMS)()
+        p["lat"] = []
+    lat_all = []
+    t_start = time.perf_counter_ns() + 2_000_000
+    for i in range(n_frames):
+        arrival = t_start + i * FRAME_PERIOD_NS
+        while time.perf_counter_ns() < arrival:
+            pass
+        if before_tick is not None:
+            before_tick(i)
+        for p in parts:
+            for s in range(p["K"]):
+                p["fr"][s].data = p["host_ring"][s][i % p["R"]].data_ptr()
+                p["fr"][s].on_device = 0
+                p["fr"][s].frame_index = i
+                p["fr"][s].arrival_ns = arrival
+            if p["ctx"].submit_raw(p["K"], p["fr"], p["sts"]) != 0:
+                raise RuntimeError(p["ctx"].last_error())
+        for p in parts:
+            if p["ctx"].sync_raw(p["res"]) != 0:
+                raise RuntimeError(p["ctx"].last_error())
+            p["lat"].append((time.perf_counter_ns() - arrival) / 1e6)
+        lat_all.append((time.perf_counter_ns() - arrival) / 1e6)
+    keys = ("mean_ms", "std_ms", "p50_ms", "p99_ms", "max_ms", "tail_p100_p95_ms", "flatness_p90_p10_ms")
+    out = {"all": {k: latency_summary(trim_warmup(lat_all))[k] for k in keys}}
+    for j, p in enumerate(parts):
+        out[p.get("name", f"part{j}")] = {k: latency_summary(trim_warmup(p["lat"]))[k] for k in keys}
+    return out
+
+
+def render_study(args):
+    """Single-GPU isolation of the visualisation load (the paper's Section VIII future work, asked with CUDA only).
+    While tick i is computed, the multi-layer render of tick i-1's masks runs on a second stream, either
+    time-shared (spread over every multiprocessor) or carved out (a few looping blocks on multiprocessors the
+    inference context leaves free).  Per-frame latency of the inference ticks for K = 1..6."""
+    import numpy as np
+    import torch
+
+    import tt_synth
+    from paper_2402_04466_b200 import binding
+    dev = torch.device("cuda", 0)
+    wl = tt_synth.workload("cfg3").with_(overlay=False)
+    R, carve = args.ring, args.carve_sms
+    rstream = torch.cuda.Stream()
+    rows = []
+    for K in [int(x) for x in args.study_streams.split(",")]:
+        frames = [[torch.from_numpy(tt_synth.make_frame(wl.frame_kind, wl.stream_seed(s), t, wl.src_w, wl.src_h)) for t in range(R)]
+                  for s in range(K)]
+        host_ring = [[f.pin_memory() for f in fs] for fs in frames]
+        stacked = [torch.stack([frames[s][t].reshape(-1) for s in range(K)]).to(dev) for t in range(R)]   # [K][bytes] per ring index
+        out_buf = torch.empty((K, wl.src_h, wl.src_w, 4), dtype=torch.uint8, device=dev)
+        hm, wm = wl.map_hw()
+        for mode in ("none", "time-shared", "carved-out"):
+            stream = torch.cuda.Stream()
+            cfg = binding.make_config(wl, max_streams=K, cuda_stream=stream.cuda_stream, reserved_sms=carve if mode == "carved-out" else 0)
+            ctx = binding.Context(cfg, tt_synth.make_weights(wl))
+            part = {"name": "inference", "ctx": ctx, "states": [ctx.state_create() for _ in range(K)], "host_ring": host_ring, "K": K, "R": R}
+            state = {"masks": None}
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            render_ms = []
+
+            def before_tick(i):
+                # the masks of the previous tick are rendered while this tick is computed
+                if mode == "none" or i == 0:
+                    return
+                res0 = part["res"][0]
+                masks = binding.device_tensor(res0.masks_dev, (K, wl.n_tools, hm, wm), np.uint8)
+                timed = (i % 16 == 1)
+                with torch.cuda.stream(rstream):
+                    if timed:
+                        ev0.record()
+                    binding.render_layers(stacked[(i - 1) % R], wl.src_w, wl.src_h, wl.src_pitch, masks, wl.palette, args.render_layers,
+                                          carve_ctas=carve if mode == "carved-out" else 0, stream=rstream, out=out_buf)
+                    if timed:
+                        ev1.record()
+                        state["pending"] = True
+
+            def harvest():
+                if state.get("pending"):
+                    ev1.synchronize()
+                    render_ms.append(ev0.elapsed_time(ev1))
+                    state["pending"] = False
+
+            # harvest the timed render of the previous period right at the next arrival (it has long finished)
+            def hook(i):
+                harvest()
+                before_tick(i)
+
+            lat = paced_multi([part], args.study_frames, before_tick=hook)
+            torch.cuda.synchronize()
+            harvest()
+            ent = {"streams": K, "mode": mode, **lat["inference"]}
+            if render_ms:
+                ent["render_ms_mean"] = sum(render_ms) / len(render_ms)
+                ent["render_ms_max"] = max(render_ms)
+            rows.append(ent)
+            ctx.destroy()
+    print(json.dumps({"study": "render isolation", "workload": describe(wl, 0).replace("K=0 ", ""), "render_layers": args.render_layers,
+                      "carved_out_sms": carve, "frames_per_stream": args.study_frames, "rows": rows}))
+    return 0
+
+
+def hetero_study(args):
+    """Two different models on one GPU (the paper's heterogeneous experiment, Section VI, Table II): the recurrent
+    tool-tracking model and a feed-forward segmentation model, alone and together (each context on its own CUDA
+    stream, both submitted every period)."""
+    import torch
+
+    import tt_synth
+    from paper_2402_04466_b200 import binding
+    dev = torch.device("cuda", 0)
+    R = args.ring
+    specs = {"tool-tracking (recurrent)": (tt_synth.workload("cfg2"), args.hetero_k),
+             "segmentation (feed-forward)": (tt_synth.workload("cfg2-ff"), args.hetero_k)}
+
+    def build(name, shared_stream=None):
+        wl, K = specs[name]
+        stream = shared_stream or torch.cuda.Stream()
+        ctx = binding.Context(binding.make_config(wl, max_streams=K, cuda_stream=stream.cuda_stream), tt_synth.make_weights(wl))
+        host_ring = [[torch.from_numpy(tt_synth.make_frame(wl.frame_kind, wl.stream_seed(s), t, wl.src_w, wl.src_h)).pin_memory()
+                      for t in range(R)] for s in range(K)]
+        return {"name": name, "ctx": ctx, "states": [ctx.state_create() for _ in range(K)], "host_ring": host_ring, "K": K, "R": R,
+                "_stream": stream}
+
+    rows = []
+    for name in specs:
+        p = build(name)
+        rows.append({"setup": "alone", **{name: paced_multi([p], args.study_frames)[name]}})
+        p["ctx"].destroy()
+    parts = [build(n) for n in specs]
+    lat = paced_multi(parts, args.study_frames)
+    rows.append({"setup": "together, one CUDA stream per model", **lat})
+    for p in parts:
+        p["ctx"].destroy()
+    one = torch.cuda.Stream()
+    parts = [build(n, one) for n in specs]
+    lat = paced_multi(parts, args.study_frames)
+    rows.append({"setup": "together, both models on one CUDA stream (serialised)", **lat})
+    for p in parts:
+        p["ctx"].destroy()
+    print(json.dumps({"study": "heterogeneous models", "streams_per_model": args.hetero_k, "frames_per_stream": args.study_frames,
+                      "models": {n: describe(w, k) for n, (w, k) in specs.items()}, "rows": rows}))
+    return 0
+
+
+def multi_model_study(args):
+    """Three models per frame (the paper's Multi-AI application, Section III-B): three feed-forward encoder/head sets
+    with different weights read the same frame; latency = arrival -> all three results on the host."""
+    import torch
+
+    import tt_synth
+    from paper_2402_04466_b200 import binding
+    R = args.ring
+    base = tt_synth.workload("cfg2-ff")
+    wls = [base.with_(name=f"model{j}", seed=base.seed + 31 * (j + 1)) for j in range(3)]
+    host_ring = [[torch.from_numpy(tt_synth.make_frame(base.frame_kind, base.stream_seed(0), t, base.src_w, base.src_h)).pin_memory()
+                  for t in range(R)]]
+
+    def build(wl, stream):
+        ctx = binding.Context(binding.make_config(wl, max_streams=1, cuda_stream=stream.cuda_stream), tt_synth.make_weights(wl))
+        return {"name": wl.name, "ctx": ctx, "states": [ctx.state_create()], "host_ring": host_ring, "K": 1, "R": R}
+
+    rows = []
+    for setup, streams in (("three CUDA streams (concurrent branches)", [torch.cuda.Stream() for _ in range(3)]),
+                           ("one CUDA stream (serialised)", [torch.cuda.Stream()] * 3)):
+        parts = [build(w, s) for w, s in zip(wls, streams)]
+        lat = paced_multi(parts, args.study_frames)
+        rows.append({"setup": setup, **lat})
+        for p in parts:
+            p["ctx"].destroy()
+    p = build(wls[0], torch.cuda.Stream())
+    rows.append({"setup": "one model alone", **paced_multi([p], args.study_frames)})
+    p["ctx"].destroy()
+    print(json.dumps({"study": "three models per frame", "model": describe(base, 1), "frames_per_stream": args.study_frames, "rows": rows}))
+    return 0
+
+
 # -------------------------------------------------------------------------------- GPU arm
 def stage_table(wl, K, stage_sum, steps, peaks):
     """Per-stage device time, achieved rate and fraction of the roof that bounds the stage."""
@@ -698,11 +892,24 @@ def main():
                     help="timed ticks of the scale-sweep configuration (cfg4, K=8) reported as target_config (0: skip)")
     ap.add_argument("--target-sweeps", type=int, default=1, help="also sweep the stream count at both sizes (0: skip)")
     ap.add_argument("--target-paced-frames", type=int, default=120, help="frames per stream of every sweep point's paced run")
+    ap.add_argument("--study", default="", choices=["", "render", "hetero", "multi-model"],
+                    help="run one of the latency studies instead of the benchmark line (1 GPU)")
+    ap.add_argument("--study-frames", type=int, default=300, help="paced frames per stream and setting of a study")
+    ap.add_argument("--study-streams", default="1,2,3,4,5,6", help="stream counts of the render study")
+    ap.add_argument("--render-layers", type=int, default=8)
+    ap.add_argument("--carve-sms", type=int, default=16, help="multiprocessors given to the carved-out render load")
+    ap.add_argument("--hetero-k", type=int, default=3, help="streams per model in the heterogeneous study")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
         return run_reference(args)
+    if args.study == "render":
+        return render_study(args)
+    if args.study == "hetero":
+        return hetero_study(args)
+    if args.study == "multi-model":
+        return multi_model_study(args)
     return run_ours(args)
 
 

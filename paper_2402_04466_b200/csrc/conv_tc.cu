@@ -44,13 +44,16 @@ constexpr int MAX_K_ITERS = 9 * 16;                // 9 taps x up to 16 channel 
 // PAIR: two CTAs of a cluster work on two neighbouring M-tiles with one MMA of 256 rows
 // (cta_group::2).  Each CTA then stages its own activation box and only its own half of the
 // weight slab's rows, so a stage holds a third less and the ring is half as deep again.
-template <int BLOCK_N, int SLAB_C, bool PAIR = false>
+// CTAS: blocks per multiprocessor the configuration is sized for.  The small encoder layers are
+// bound by the latency of their single-thread issue chains, not by bandwidth or arithmetic: two
+// blocks per multiprocessor (half the ring each) run two such chains side by side.
+template <int BLOCK_N, int SLAB_C, bool PAIR = false, int CTAS = 1>
 struct TcCfg {
   static constexpr int A_BYTES = BLOCK_M * SLAB_C * 2;
   static constexpr int B_ROWS = PAIR ? BLOCK_N / 2 : BLOCK_N;     // weight rows staged by one CTA
   static constexpr int B_BYTES = B_ROWS * SLAB_C * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES_RAW = (192 * 1024) / STAGE_BYTES;
+  static constexpr int STAGES_RAW = ((CTAS == 2 ? 104 : 192) * 1024) / STAGE_BYTES;
   static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
   static constexpr int TMEM_COLS = 2 * BLOCK_N < 32 ? 32 : 2 * BLOCK_N;
   static constexpr int BAR_BYTES = 256;
@@ -72,9 +75,11 @@ __device__ __forceinline__ float fast_sigmoid(float z) { return fmaf(0.5f, fast_
 
 
 // ------------------------------------------------------------------------------------ kernel
-template <int BLOCK_N, int SLAB_C, int EPI, bool PAIR>
-__global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_constant__ ConvTcParams p) {
-  using Cfg = TcCfg<BLOCK_N, SLAB_C, PAIR>;
+template <int BLOCK_N, int SLAB_C, int EPI, bool PAIR, int CTAS = 1>
+__global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_constant__ ConvTcParams p) {
+  using Cfg = TcCfg<BLOCK_N, SLAB_C, PAIR, CTAS>;
+  static_assert(CTAS == 1 || (CTAS == 2 && !PAIR && Cfg::TMEM_COLS <= 256 && Cfg::SMEM_BYTES <= 112 * 1024),
+                "two blocks per multiprocessor must fit its shared and tensor memory");
   constexpr int STAGES = Cfg::STAGES;
   constexpr uint32_t LAYOUT = SLAB_C == 64 ? 2u : 4u;
   constexpr uint32_t SBO = 8u * SLAB_C * 2u;
@@ -391,14 +396,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const __grid_con
   }
 }
 
-template <int BLOCK_N, int SLAB_C, int EPI>
+template <int BLOCK_N, int SLAB_C, int EPI, int CTAS = 1>
 cudaError_t launch_cfg(const ConvTcParams& p, int sm_count, cudaStream_t s) {
-  using Cfg = TcCfg<BLOCK_N, SLAB_C>;
-  auto kern = conv_tc_kernel<BLOCK_N, SLAB_C, EPI, false>;
+  using Cfg = TcCfg<BLOCK_N, SLAB_C, false, CTAS>;
+  auto kern = conv_tc_kernel<BLOCK_N, SLAB_C, EPI, false, CTAS>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int total_tiles = p.K * p.tiles_x * p.tiles_y * p.n_tiles_n;
-  const int grid = total_tiles < sm_count ? total_tiles : sm_count;
+  const int slots = CTAS * sm_count;
+  const int grid = total_tiles < slots ? total_tiles : slots;
   return launch_kernel(kern, grid, TC_THREADS, Cfg::SMEM_BYTES, s, p, p.pdl != 0);
 }
 
@@ -444,6 +450,12 @@ cudaError_t launch_shape(const ConvTcParams& p, int sm_count, cudaStream_t s) {
   if (p.pair) {
     if (p.slab_c == 64 && p.block_n == 256) return launch_pair<256, 64, EPI>(p, sm_count, s);
     return cudaErrorInvalidValue;
+  }
+  if (EPI == TC_EPI_RELU_BF16 && p.two_per_sm && p.block_n <= 128) {
+    if (p.slab_c == 64 && p.block_n == 128) return launch_cfg<128, 64, TC_EPI_RELU_BF16, 2>(p, sm_count, s);
+    if (p.slab_c == 64 && p.block_n == 64) return launch_cfg<64, 64, TC_EPI_RELU_BF16, 2>(p, sm_count, s);
+    if (p.slab_c == 32 && p.block_n == 128) return launch_cfg<128, 32, TC_EPI_RELU_BF16, 2>(p, sm_count, s);
+    if (p.slab_c == 32 && p.block_n == 64) return launch_cfg<64, 32, TC_EPI_RELU_BF16, 2>(p, sm_count, s);
   }
   if (p.slab_c == 64) {
     if (p.block_n == 256) return launch_cfg<256, 64, EPI>(p, sm_count, s);

@@ -151,6 +151,7 @@ struct tt_ctx {
   std::vector<TickGraph> graphs;
   bool graphs_off = false;
   bool cta_pairs = false;           // TT_OPT_CTA_PAIRS
+  bool enc_two_per_sm = true;       // !TT_OPT_ENC_ONE_PER_SM
   bool feed_forward = false;        // TT_OPT_FEED_FORWARD: no recurrent cell, the heads read the encoder output
   const uint8_t** frame_tab_dev[2] = {nullptr, nullptr};   // device, [TT_MAX_STREAMS] pointers per slot
   const uint8_t** frame_tab_host[2] = {nullptr, nullptr};  // pinned staging of the same
@@ -364,18 +365,21 @@ tt_status pack_tc(tt_ctx* ctx, TcLayer* L, const float* w, const float* b, int c
   return TT_OK;
 }
 
-int pick_block_n(const TcLayer& L, int m_tiles, int sm_count) {
+// two_per_sm: tiles up to 128 wide run two blocks per multiprocessor (encoder layers)
+int pick_block_n(const TcLayer& L, int m_tiles, int sm_count, bool two_per_sm) {
   const int bns[3] = {64, 128, 256};
   int best = -1;
   double best_cost = 0;
   for (int i = 0; i < 3; ++i) {
     if (!L.has_b[i]) continue;
     const long tiles = (long)m_tiles * (L.cout / bns[i]);
-    const long waves = (tiles + sm_count - 1) / sm_count;
+    const int per_sm = (two_per_sm && bns[i] <= 128) ? 2 : 1;
+    const long slots = (long)per_sm * sm_count;
+    const long waves = (tiles + slots - 1) / slots;
     // Time of a tile: its main loop is paced by the thread that issues the MMAs (about 600 cycles
     // per K slab whatever the width) until the tensor pipe itself needs longer (2 cycles per
-    // column and K slab of 64 at 128 rows).
-    const double cost = (double)waves * std::max(600.0, 2.5 * bns[i]);
+    // column and K slab of 64 at 128 rows, shared by the blocks of a multiprocessor).
+    const double cost = (double)waves * std::max(600.0, 2.5 * bns[i] * per_sm);
     if (best < 0 || cost < best_cost - 1e-9 || (std::fabs(cost - best_cost) < 1e-9 && bns[i] > bns[best])) {
       best = i;
       best_cost = cost;
@@ -511,6 +515,7 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
   bind_slot(ctx, 0);
   ctx->graphs_off = c.options[TT_OPT_PLAIN_LAUNCHES] != 0;
   ctx->cta_pairs = c.options[TT_OPT_CTA_PAIRS] != 0;
+  ctx->enc_two_per_sm = c.options[TT_OPT_ENC_ONE_PER_SM] == 0;
   ctx->feed_forward = c.options[TT_OPT_FEED_FORWARD] != 0;
   const bool no_post_tc = c.options[TT_OPT_NO_POST_TC] != 0;
 
@@ -735,17 +740,18 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
       TT_CUDA(ctx, launch_conv_simt(q, s));
       if ((ms_ = mark_stage(ctx, TT_STAGE_ENC0, 1)) != TT_OK) return ms_;
     }
-    auto fill_common = [&](ConvTcParams& q, const TcLayer& L, int Ho, int Wo) -> tt_status {
+    auto fill_common = [&](ConvTcParams& q, const TcLayer& L, int Ho, int Wo, bool encoder) -> tt_status {
       std::memcpy(q.maps_a, L.maps_a, sizeof(q.maps_a));
       q.slab_c = L.slab_c; q.stride = L.stride; q.K = K; q.Ho = Ho; q.Wo = Wo;
       q.tiles_x = (Wo + 15) / 16; q.tiles_y = (Ho + 7) / 8;
-      const int bi = pick_block_n(L, K * q.tiles_x * q.tiles_y, ctx->sm_count);
+      const int bi = pick_block_n(L, K * q.tiles_x * q.tiles_y, ctx->sm_count, encoder && ctx->enc_two_per_sm);
       if (bi < 0) return fail(ctx, TT_ERR_UNSUPPORTED, "no tensor-core tile shape fits this layer");
       const int bns[3] = {64, 128, 256};
       q.block_n = bns[bi]; q.map_b = L.map_b[bi]; q.n_tiles_n = L.cout / q.block_n;
       // on request 256-wide tiles run on CTA pairs: each CTA stages its own activation box and half of the weight slab
       q.pair = (bi == 2 && L.slab_c == 64 && L.has_b[1] && ctx->cta_pairs && K * q.tiles_x * q.tiles_y >= 2) ? 1 : 0;
       if (q.pair) q.map_b = L.map_b[1];
+      q.two_per_sm = (encoder && ctx->enc_two_per_sm) ? 1 : 0;
       q.cout = L.cout; q.bias = L.b; q.status = ctx->status_dev; q.wait_limit = ctx->wait_limit;
       q.n_prod = 3;
       q.pdl = ctx->profiling ? 0 : 1;
@@ -754,7 +760,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
     for (int l = 1; l < ctx->n_enc; ++l) {
       const TcLayer& L = ctx->tc_enc[l];
       ConvTcParams q{};
-      tt_status st = fill_common(q, L, ctx->lay_h[l + 1], ctx->lay_w[l + 1]);
+      tt_status st = fill_common(q, L, ctx->lay_h[l + 1], ctx->lay_w[l + 1], true);
       if (st != TT_OK) return st;
       q.n_src = 1; q.slabs[0] = L.cin0 / L.slab_c; q.slabs[1] = 0; q.img0 = ident; q.img1 = ident;
       q.epilogue = TC_EPI_RELU_BF16; q.out = reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[l]);
@@ -764,7 +770,7 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
     if (!ctx->feed_forward) {
     const TcLayer& L = ctx->tc_lstm;
     ConvTcParams q{};
-    tt_status st = fill_common(q, L, ctx->Hm, ctx->Wm);
+    tt_status st = fill_common(q, L, ctx->Hm, ctx->Wm, false);
     if (st != TT_OK) return st;
     q.n_src = 2; q.slabs[0] = L.cin0 / L.slab_c; q.slabs[1] = L.cin1 / L.slab_c; q.img0 = ident; q.img1 = h_in;
     q.epilogue = TC_EPI_LSTM; q.c_state = ctx->c_state; q.h_f32 = ctx->h_f32; q.h_bf16 = ctx->h_bf16;

@@ -121,3 +121,22 @@ def test_overlay_is_bit_exact(cuda_device, src_wh, grid, pad, K, T):
     for k in range(K):
         ref = oracle.overlay(frames[k], masks[k], tt_synth.configs.PALETTE)
         assert np.array_equal(out[k], ref)
+
+
+@pytest.mark.parametrize("src_wh,grid,pad,K,T,layers", [((214, 120), (15, 20), 0, 2, 7, 3), ((50, 31), (7, 9), 3, 3, 4, 5),
+                                                        ((854, 480), (60, 80), 0, 1, 7, 2)])
+def test_render_layers_is_bit_exact_in_both_forms(cuda_device, src_wh, grid, pad, K, T, layers):
+    """The multi-layer visualisation load against the oracle's layer-by-layer blend: the time-shared form (a block
+    per 1024 pixels) and the carved-out form (a few looping blocks) must give the same bytes."""
+    (sw, sh), (hm, wm) = src_wh, grid
+    frames = RNG.integers(0, 256, (K, sh, sw, 3), dtype=np.uint8)
+    masks = (RNG.random((K, T, hm, wm)) < 0.4).astype(np.uint8)
+    pitch = 3 * sw + pad
+    src = _frames_to_dev(frames, pitch, cuda_device)
+    m_dev = torch.from_numpy(masks).to(cuda_device)
+    shared = binding.render_layers(src, sw, sh, pitch, m_dev, tt_synth.configs.PALETTE, layers).cpu().numpy()
+    carved = binding.render_layers(src, sw, sh, pitch, m_dev, tt_synth.configs.PALETTE, layers, carve_ctas=3).cpu().numpy()
+    for k in range(K):
+        ref = oracle.render_layers(frames[k], masks[k], tt_synth.configs.PALETTE, layers)
+        assert np.array_equal(shared[k], ref)
+        assert np.array_equal(carved[k], ref)

@@ -84,3 +84,5 @@ def test_stage_level_calls_refuse_misaligned_or_oversized_arguments_on_the_host(
     assert b"dst_dev" in lib.tt_last_error(None)
     assert lib.tt_overlay(A, 1, 0, 8, 8, 24, A + 0x10000, 4, 20000, 4, pal, A + 0x20000, None) == 1
     assert lib.tt_debug_expire_wait(None, 1000) == 1
+    assert lib.tt_render_layers(A, 1, 0, 8, 8, 24, A + 0x10000, 4, 4, 4, pal, 0, 0, A + 0x20000, None) == 1      # layers < 1
+    assert lib.tt_render_layers(A, 1, 0, 8, 8, 24, A + 0x10000, 4, 4, 4, pal, 2, 0, A + 0x20001, None) == 1      # misaligned output
