@@ -350,7 +350,7 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
               h_new[jj] = fast_sigmoid(go) * fast_tanh(c_new[jj]);
             }
             st_global_v8(p.c_state + so + ck * 8, c_new);
-            st_global_v8(p.h_f32 + so + ck * 8, h_new);
+            if (p.h_f32) st_global_v8(p.h_f32 + so + ck * 8, h_new);
             // bf16 shadow of h': 8 values are half a sector, so two neighbouring chunks leave together
             const int hq = (ck & 1) * 4;
             hb[hq + 0] = pack_bf16(h_new[0], h_new[1]);

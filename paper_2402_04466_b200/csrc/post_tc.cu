@@ -10,14 +10,14 @@
 // slabs (128-byte swizzle) through a ring of stages.  The stage is bound by HBM: the tensor work
 // and the per-pixel epilogue (bias, sigmoid, threshold, outputs) are far below the copy time.
 //
-// Warp roles (192 threads, two blocks per multiprocessor): warp 0 = TMA producer (one lane),
+// Warp roles (192 threads, three blocks per multiprocessor): warp 0 = TMA producer (one lane),
 // warp 1 = tensor-memory allocation and MMA issue (one lane), warps 2..5 = epilogue, one thread per
 // pixel of the tile (tensor-memory lane = pixel).  Per tile every epilogue warp reduces its 32
 // pixels' statistics (mask count, sum x, sum y by integer warp reductions; probability or
-// confidence-head sums in a fixed shuffle order, then to fixed point) and adds them to the block's
-// accumulators in shared memory; these reach the per-stream accumulators in global memory through
-// integer atomics when the block moves on to another stream or ends, and the block that completes
-// a stream forms its result record and zeroes the accumulators again.  Integer additions commute,
+// confidence-head sums in a fixed shuffle order, then to fixed point); lane t keeps tool t's running
+// sums in registers.  When the block moves on to another stream or ends, the warps' sums meet in
+// shared memory and reach the per-stream accumulators in global memory through integer atomics;
+// the block that completes a stream forms its result record and zeroes the accumulators again.  Integer additions commute,
 // and the floating-point partial sums are formed over fixed groups of 32 pixels of one stream, so
 // a stream's results do not depend on what else shares the launch.
 // Every barrier wait is bounded (see tc_ptx.cuh).
@@ -30,7 +30,7 @@ namespace {
 using namespace tc;
 
 constexpr int PT_THREADS = 192;
-constexpr int PT_STAGES = 5;
+constexpr int PT_STAGES = 3;                      // slabs in flight per block (a tile is hidden / 64 slabs)
 constexpr int PT_SLAB_BYTES = 128 * 64 * 2;        // 128 pixels x 64 channels bf16
 constexpr int PT_WSLAB_BYTES = 16 * 64 * 2;        // 16 weight rows x 64 channels bf16
 constexpr int PT_MAX_SLABS = 8;                    // hidden <= 512
@@ -66,7 +66,7 @@ __device__ __forceinline__ float sigmoid_fast(float z) { return __fdividef(1.0f,
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-__global__ void __launch_bounds__(PT_THREADS, 2) post_tc_kernel(const __grid_constant__ PostTcParams p) {
+__global__ void __launch_bounds__(PT_THREADS, 3) post_tc_kernel(const __grid_constant__ PostTcParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* s_w = smem + PT_STAGES * PT_SLAB_BYTES;                       // [kslabs] weight slabs, 1024-byte aligned
@@ -220,6 +220,22 @@ __global__ void __launch_bounds__(PT_THREADS, 2) post_tc_kernel(const __grid_con
       epi_bar();
     };
 
+    // Lane t < T of every epilogue warp carries tool t's running sums for the stream the block is
+    // working on (mask count, sum x, sum y, and the fixed-point sum of probabilities or of the
+    // confidence-head column); they meet in the block's shared accumulators only when the block
+    // moves on to another stream or ends.
+    long long r_cnt = 0, r_sx = 0, r_sy = 0, r_sum = 0;
+    auto spill = [&]() {
+      if (lane < T) {
+        if (p.conf_mode == TT_CONF_MEAN_SIGMOID) atomicAdd(s_acc + 8 + lane * 4 + 3, (unsigned long long)r_sum);
+        else atomicAdd(s_acc + lane, (unsigned long long)r_sum);
+        atomicAdd(s_acc + 8 + lane * 4 + 0, (unsigned long long)r_cnt);
+        atomicAdd(s_acc + 8 + lane * 4 + 1, (unsigned long long)r_sx);
+        atomicAdd(s_acc + 8 + lane * 4 + 2, (unsigned long long)r_sy);
+      }
+      r_cnt = r_sx = r_sy = r_sum = 0;
+    };
+
     uint32_t acc_phase = 0;
     int acc = 0;
     int cur_n = t_begin < t_end ? t_begin / tpi : 0, tiles_done = 0;
@@ -227,6 +243,7 @@ __global__ void __launch_bounds__(PT_THREADS, 2) post_tc_kernel(const __grid_con
     for (int tile = t_begin; tile < t_end; ++tile) {
       const int n = tile / tpi, pix0 = (tile - n * tpi) << 7;
       if (n != cur_n) {
+        spill();
         flush(cur_n, tiles_done);
         cur_n = n;
         tiles_done = 0;
@@ -246,6 +263,7 @@ __global__ void __launch_bounds__(PT_THREADS, 2) post_tc_kernel(const __grid_con
       const int pix = pix0 + quarter * 32 + lane;
       const bool live = pix < plane;
       const int px = live ? pix % p.Wm : 0, py = live ? pix / p.Wm : 0;
+      const size_t o0 = (size_t)n * T * plane + pix;     // tool t's element: + t * plane
       uint32_t bits = 0;
 #pragma unroll
       for (int t = 0; t < TT_MAX_TOOLS; ++t) {
@@ -254,7 +272,7 @@ __global__ void __launch_bounds__(PT_THREADS, 2) post_tc_kernel(const __grid_con
           const float pr = sigmoid_fast(z);
           const bool m = live && (z > p.zthr);
           if (live) {
-            const size_t o = ((size_t)n * T + t) * plane + pix;
+            const size_t o = o0 + (size_t)t * plane;
             p.logits[o] = z;
             p.probs[o] = pr;
             p.masks[o] = m ? 1 : 0;
@@ -274,25 +292,17 @@ __global__ void __launch_bounds__(PT_THREADS, 2) post_tc_kernel(const __grid_con
             for (int d = 16; d > 0; d >>= 1) g += __shfl_xor_sync(0xffffffffu, g, d);
             s1 = __float2ll_rn(g * PT_FIX_SCALE);
           }
-          if (lane == 0) {
-            if (p.conf_mode == TT_CONF_MEAN_SIGMOID) {
-              atomicAdd(s_acc + 8 + t * 4 + 3, (unsigned long long)s1);
-            } else {
-              atomicAdd(s_acc + t, (unsigned long long)s1);
-            }
-            if (c1) {
-              atomicAdd(s_acc + 8 + t * 4 + 0, (unsigned long long)c1);
-              atomicAdd(s_acc + 8 + t * 4 + 1, (unsigned long long)x1);
-              atomicAdd(s_acc + 8 + t * 4 + 2, (unsigned long long)y1);
-            }
-          }
+          if (lane == t) { r_cnt += c1; r_sx += x1; r_sy += y1; r_sum += s1; }
         }
       }
       if (p.bits && live) p.bits[(size_t)n * plane + pix] = (uint8_t)bits;
       tiles_done += 1;
     }
     // hand on what the block has gathered (after a wait that ran out the tick's results are void anyway)
-    if (ok && t_begin < t_end) flush(cur_n, tiles_done);
+    if (ok && t_begin < t_end) {
+      spill();
+      flush(cur_n, tiles_done);
+    }
   }
 
   // ------------------------------------------------------------------------------- teardown
@@ -320,7 +330,7 @@ cudaError_t launch_post_tc(const PostTcParams& p, int sm_count, cudaStream_t s) 
   if (e != cudaSuccess) return e;
   const int plane = p.Hm * p.Wm;
   const int total = p.K * ((plane + 127) / 128);
-  const int grid = total < 2 * sm_count ? total : 2 * sm_count;
+  const int grid = total < 3 * sm_count ? total : 3 * sm_count;
   return launch_kernel(post_tc_kernel, grid, PT_THREADS, (size_t)smem, s, p, p.pdl != 0);
 }
 

@@ -773,7 +773,9 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
     tt_status st = fill_common(q, L, ctx->Hm, ctx->Wm, false);
     if (st != TT_OK) return st;
     q.n_src = 2; q.slabs[0] = L.cin0 / L.slab_c; q.slabs[1] = L.cin1 / L.slab_c; q.img0 = ident; q.img1 = h_in;
-    q.epilogue = TC_EPI_LSTM; q.c_state = ctx->c_state; q.h_f32 = ctx->h_f32; q.h_bf16 = ctx->h_bf16;
+    // with the heads on the tensor cores nothing on the path reads an fp32 copy of h': its consumers (the next
+    // step's convolution and the heads) take the bf16 copy, so only that copy is written
+    q.epilogue = TC_EPI_LSTM; q.c_state = ctx->c_state; q.h_f32 = ctx->use_post_tc ? nullptr : ctx->h_f32; q.h_bf16 = ctx->h_bf16;
     q.c_idx = c_idx; q.h_out_idx = h_out; q.hidden = ctx->Ch;
     TT_CUDA(ctx, launch_conv_tc(q, ctx->sm_count, s));
     if ((ms_ = mark_stage(ctx, TT_STAGE_CONVLSTM, 1)) != TT_OK) return ms_;
@@ -913,7 +915,10 @@ tt_status tt_state_export(tt_ctx* ctx, tt_state* st, float* h_host, float* c_hos
   const int plane = ctx->Hm * ctx->Wm;
   const size_t n = (size_t)ctx->Ch * plane;
   if (ctx->bf16) {
-    TT_CUDA(ctx, launch_nhwc_to_nchw_f32(ctx->h_f32 + (size_t)st->slot * n, ctx->dbg_tmp, ctx->Ch, plane, ctx->stream));
+    if (ctx->use_post_tc)   // h' exists as its bf16 copy only; every bf16 value is an fp32 value
+      TT_CUDA(ctx, launch_nhwc_bf16_to_nchw_f32(ctx->h_bf16 + ((size_t)st->slot * 2 + st->half) * n, ctx->dbg_tmp, ctx->Ch, plane, ctx->stream));
+    else
+      TT_CUDA(ctx, launch_nhwc_to_nchw_f32(ctx->h_f32 + (size_t)st->slot * n, ctx->dbg_tmp, ctx->Ch, plane, ctx->stream));
     TT_CUDA(ctx, cudaMemcpyAsync(h_host, ctx->dbg_tmp, n * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
     TT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     TT_CUDA(ctx, launch_nhwc_to_nchw_f32(ctx->c_state + (size_t)st->slot * n, ctx->dbg_tmp, ctx->Ch, plane, ctx->stream));

@@ -136,7 +136,7 @@ struct ConvTcParams {
   __nv_bfloat16* out;       // [K][Ho][Wo][cout]
   // LSTM epilogue
   float* c_state;           // [slots][Hm][Wm][Ch] in place
-  float* h_f32;             // [slots][Hm][Wm][Ch]
+  float* h_f32;             // [slots][Hm][Wm][Ch], or null: h' is written as its bf16 copy only
   __nv_bfloat16* h_bf16;    // [slots*2][Hm][Wm][Ch]
   IdxMap c_idx, h_out_idx;  // slot, slot*2+half
   int32_t hidden;

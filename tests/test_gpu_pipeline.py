@@ -611,6 +611,44 @@ def test_two_models_in_the_same_tick_match_their_solo_runs(cuda_device):
     cb.destroy()
 
 
+def test_three_models_on_the_same_frame_as_concurrent_branches(cuda_device):
+    """A multi-model stream (the paper's Multi-AI application, Section III-B: three models fed by one video): three
+    feed-forward encoder/head sets with different weights read the same frame, each context on its own CUDA stream so
+    that the three branches run concurrently.  Every model must match the oracle and its own solo run bit for bit."""
+    base = tt_synth.workload("cfg1-ff-gain").with_(src_w=214, src_h=120, net_w=176, net_h=136)
+    wls = [base.with_(name=f"multi{j}", seed=base.seed + 31 * (j + 1)) for j in range(3)]
+    n = 3
+    frames = tt_synth.make_frames(base.frame_kind, base.stream_seed(0), n, base.src_w, base.src_h)
+    dev_frames = [torch.from_numpy(f).to(cuda_device) for f in frames]
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    models = []
+    for wl, s in zip(wls, streams):
+        w = tt_synth.make_weights(wl)
+        ctx = binding.Context(binding.make_config(wl, max_streams=1, cuda_stream=s.cuda_stream), w)
+        models.append((wl, w, ctx, ctx.state_create()))
+    assert not np.array_equal(models[0][1]["head_w"], models[1][1]["head_w"])      # three different models
+    torch.cuda.synchronize()
+    together = []
+    for t in range(n):
+        for _, _, ctx, st in models:
+            ctx.submit_frames([dev_frames[t]], [st], frame_index=t)                   # all three in flight
+        row = []
+        for wl, w, ctx, st in models:
+            (res,) = ctx.sync()
+            ref = oracle.OraclePipeline(wl, w).step(frames[t], want_overlay=False)
+            band = max(1e-3, BAND_REL * float(np.sqrt(np.mean(ref.z.astype(np.float64) ** 2))))
+            _compare_frame(ctx, st, res, ref, TOL_OUT, band, tag=f"{wl.name} t={t}", tol_mid=TOL_MID_PLAIN)
+            row.append((ctx.fetch_probs(res), res["conf"].copy(), res["count"].copy()))
+        together.append(row)
+    for j, (wl, w, ctx, st) in enumerate(models):
+        for t in range(n):                                                            # the same model alone
+            ctx.submit_frames([dev_frames[t]], [st], frame_index=t)
+            (res,) = ctx.sync()
+            a = (ctx.fetch_probs(res), res["conf"].copy(), res["count"].copy())
+            assert all(np.array_equal(x, y) for x, y in zip(a, together[t][j]))
+        ctx.destroy()
+
+
 def test_host_side_sync_timeout_leaves_the_submit_in_flight(cuda_device):
     """Failure detection on the host: with sync_timeout_ns = 1 us the first tt_sync of a scale-sweep-sized tick
     gives up with TT_ERR_TIMEOUT (nothing is lost, the submit stays in flight); repeating the call until it
