@@ -102,10 +102,14 @@ def stage_work(wl, K):
             out[f"enc{l}"] = {"bound": "tensor", "flops": flops, "bytes": in_bytes + out_bytes}
         h, w, cin = ho, wo, co
     ch = wl.hidden
-    out["convlstm"] = {"bound": "tensor" if wl.precision == "bf16" else "alu",
-                       "flops": 2.0 * K * plane * 4 * ch * 9 * (cin + ch),
-                       "bytes": K * plane * (cin * act_bytes + ch * act_bytes + 8 * ch + 4 * ch + 2 * ch)}
-    out["postprocess"] = {"bound": "hbm", "bytes": K * plane * (4 * ch + wl.n_tools * 9 + 1)}
+    # on the bf16 path the heads run on the tensor cores from the bf16 copy of h' when the hidden width is a
+    # multiple of 64 and the map has at least 128 pixels; the ConvLSTM then writes no fp32 copy of h'
+    heads_bf16 = wl.precision == "bf16" and ch % 64 == 0 and ch <= 512 and plane >= 128
+    if getattr(wl, "recurrent", True):
+        out["convlstm"] = {"bound": "tensor" if wl.precision == "bf16" else "alu",
+                           "flops": 2.0 * K * plane * 4 * ch * 9 * (cin + ch),
+                           "bytes": K * plane * (cin * act_bytes + ch * act_bytes + 8 * ch + (0 if heads_bf16 else 4 * ch) + 2 * ch)}
+    out["postprocess"] = {"bound": "hbm", "bytes": K * plane * ((2 if heads_bf16 else 4) * ch + wl.n_tools * 9 + 1)}
     if wl.overlay:
         out["overlay"] = {"bound": "hbm", "bytes": K * (7 * wl.src_w * wl.src_h + plane)}
     return out

@@ -63,6 +63,8 @@ typedef enum {
                                 multiprocessors (the single-GPU isolation the paper leaves as future work, Section VIII) */
   TT_OPT_ENC_ONE_PER_SM = 5, /* run the tensor-core encoder layers with one block per multiprocessor instead of two
                                 (for A/B measurements) */
+  TT_OPT_NO_HALO = 6,        /* ConvLSTM fetches one activation box per tap instead of one haloed patch per channel
+                                slab (for A/B measurements) */
   TT_OPT_NO_POST_TC = 3      /* bf16 path: post-process from the fp32 hidden state, not from its bf16 copy on the
                                 tensor cores (for A/B measurements; not available for feed-forward models) */
 } tt_option;

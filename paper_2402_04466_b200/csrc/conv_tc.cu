@@ -59,6 +59,17 @@ struct TcCfg {
   static constexpr int BAR_BYTES = 256;
   static constexpr int TAB_BYTES = MAX_K_ITERS * 16 + 4 * TT_MAX_STREAMS * 4;   // iteration table + image index maps
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + TAB_BYTES + 1024 /*alignment slack*/;
+  // Halo mode (stride 1, 64-channel slabs): the activation ring holds haloed patches, one per
+  // channel slab: 18 rows x 16 pixels x 64 channels for an 8 x 16 output patch (10 of the 16
+  // columns are needed; a row pitch of 16 pixels = 2048 bytes keeps every 8-pixel operand group
+  // of every tap at the same phase of the 1024-byte swizzle pattern).  The weight ring holds one
+  // [BLOCK_N][64] slab per tap.
+  static constexpr int HALO_PITCH = 16, HALO_ROWS = 18;
+  static constexpr int HALO_A_BYTES = HALO_ROWS * HALO_PITCH * SLAB_C * 2;   // 36864
+  static constexpr int HALO_A_STAGES = 2;
+  static constexpr int HALO_B_RAW = (204 * 1024 - HALO_A_STAGES * HALO_A_BYTES) / B_BYTES;
+  static constexpr int HALO_B_STAGES = HALO_B_RAW > 8 ? 8 : HALO_B_RAW;
+  static constexpr int HALO_SMEM_BYTES = HALO_B_STAGES * B_BYTES + HALO_A_STAGES * HALO_A_BYTES + BAR_BYTES + TAB_BYTES + 1024;
   static_assert(STAGES >= N_PROD, "every producer needs a stage of its own");
   static_assert((TMEM_COLS & (TMEM_COLS - 1)) == 0 && TMEM_COLS <= 512, "TMEM columns must be a power of two <= 512");
   static_assert(A_BYTES % 1024 == 0 && B_BYTES % 1024 == 0, "operand tiles must keep 1024-byte alignment");
@@ -75,24 +86,33 @@ __device__ __forceinline__ float fast_sigmoid(float z) { return fmaf(0.5f, fast_
 
 
 // ------------------------------------------------------------------------------------ kernel
-template <int BLOCK_N, int SLAB_C, int EPI, bool PAIR, int CTAS = 1>
+template <int BLOCK_N, int SLAB_C, int EPI, bool PAIR, int CTAS = 1, bool HALO = false>
 __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_constant__ ConvTcParams p) {
   using Cfg = TcCfg<BLOCK_N, SLAB_C, PAIR, CTAS>;
+  static_assert(!HALO || (SLAB_C == 64 && !PAIR && CTAS == 1), "halo mode: 64-channel slabs, one block per multiprocessor");
+  constexpr int PW = HALO ? 8 : PATCH_W;           // output patch: 8 x 16 pixels in halo mode, 16 x 8 otherwise
+  constexpr int PH = HALO ? 16 : PATCH_H;
   static_assert(CTAS == 1 || (CTAS == 2 && !PAIR && Cfg::TMEM_COLS <= 256 && Cfg::SMEM_BYTES <= 112 * 1024),
                 "two blocks per multiprocessor must fit its shared and tensor memory");
-  constexpr int STAGES = Cfg::STAGES;
+  // ring depth: stages of (A + B); in halo mode the weight ring, with the activation ring of its own behind it
+  constexpr int STAGES = HALO ? Cfg::HALO_B_STAGES : Cfg::STAGES;
+  constexpr int RING_STRIDE = HALO ? Cfg::B_BYTES : Cfg::STAGE_BYTES;
+  constexpr int A_STAGES = Cfg::HALO_A_STAGES;
   constexpr uint32_t LAYOUT = SLAB_C == 64 ? 2u : 4u;
   constexpr uint32_t SBO = 8u * SLAB_C * 2u;
   constexpr uint32_t IDESC = make_idesc(PAIR ? 2 * BLOCK_M : BLOCK_M, BLOCK_N);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* bar_mem = smem + STAGES * Cfg::STAGE_BYTES;
+  uint8_t* smem_a = smem + STAGES * RING_STRIDE;               // halo mode: activation ring behind the weight ring
+  uint8_t* bar_mem = smem_a + (HALO ? A_STAGES * Cfg::HALO_A_BYTES : 0);
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(bar_mem);   // [STAGES]
   uint64_t* empty_bar = full_bar + STAGES;                     // [STAGES]
   uint64_t* tfull_bar = empty_bar + STAGES;                    // [2]
   uint64_t* tempty_bar = tfull_bar + 2;                        // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  uint64_t* afull_bar = tempty_bar + 2;                        // [2] halo mode: patch landed
+  uint64_t* aempty_bar = afull_bar + 2;                        // [2] halo mode: all nine taps have read the patch
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aempty_bar + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int4* s_tab = reinterpret_cast<int4*>(bar_mem + Cfg::BAR_BYTES);            // [k_iters] {map slot, channel offset, dx, dy}
   int* s_img = reinterpret_cast<int*>(s_tab + MAX_K_ITERS);                   // [4][TT_MAX_STREAMS]: img0, img1, c_idx, h_out_idx
@@ -150,6 +170,8 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(tfull_bar + a), 1);
       mbar_init(smem_u32(tempty_bar + a), PAIR ? 2 * EPI_WARPS : EPI_WARPS);
+      mbar_init(smem_u32(afull_bar + a), 1);
+      mbar_init(smem_u32(aempty_bar + a), 1);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -187,9 +209,46 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
     int it = prod;
     bool ok = true;
     const uint8_t* maps = reinterpret_cast<const uint8_t*>(p.maps_a);
+    if (HALO) {
+      // Iteration g = (slab, tap), slab-major: the weight slab of that tap and channel slab.  The
+      // producer that owns a slab's first tap also fetches the slab's haloed activation patch
+      // (x slabs first, then h slabs) into the activation ring, whose stage and phase follow from
+      // the running slab count.
+      const int cin_total = slabs_per_tap * SLAB_C;
+      int slab_seq0 = 0;                               // slabs of all earlier tiles of this block
+      for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
+        const int nt = tile % p.n_tiles_n;
+        const int m = tile / p.n_tiles_n;
+        const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
+        const int img_x = s_img[img], img_h = s_img[TT_MAX_STREAMS + img];
+        for (; it < k_iters; it += n_prod) {
+          const int sg = it / 9, tap = it - sg * 9;
+          if (tap == 0) {
+            const int seq = slab_seq0 + sg;
+            const uint32_t a_stage = (uint32_t)seq & 1u, a_phase = ((uint32_t)seq >> 1) & 1u;
+            ok = mbar_wait(smem_u32(aempty_bar + a_stage), a_phase ^ 1u, abort_flag, p.status, 0x900 + (int)a_stage, wait_limit);
+            if (!ok) break;
+            const int src = sg < p.slabs[0] ? 0 : 1;
+            const uint32_t ab = smem_u32(afull_bar + a_stage);
+            mbar_arrive_expect_tx(ab, Cfg::HALO_A_BYTES);
+            tma_load_4d(smem_u32(smem_a + a_stage * Cfg::HALO_A_BYTES), &p.maps_halo[src], ab, (src ? sg - p.slabs[0] : sg) * SLAB_C,
+                        tx * PW - 1, ty * PH - 1, src ? img_h : img_x);
+          }
+          ok = mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag, p.status, 0x100 + (int)stage, wait_limit);
+          if (!ok) break;
+          const uint32_t fb = smem_u32(full_bar + stage);
+          mbar_arrive_expect_tx(fb, Cfg::B_BYTES);
+          tma_load_2d(smem_u32(smem + stage * Cfg::B_BYTES), &p.map_b, fb, tap * cin_total + sg * SLAB_C, nt * BLOCK_N);
+          stage += (uint32_t)n_prod;
+          if (stage >= (uint32_t)STAGES) { stage -= STAGES; phase ^= 1u; }
+        }
+        it -= k_iters;
+        slab_seq0 += slabs_per_tap;
+      }
+    }
     // a pair's copies are counted on the leader's barriers
     const uint32_t full0c = PAIR ? map_to_cta(smem_u32(full_bar), 0u) : 0u;
-    for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
+    for (int tile = worker; tile < total_tiles && ok && !HALO; tile += n_workers) {
       const int nt = tile % p.n_tiles_n;
       // the second CTA of a pair takes the next M-tile; past the end it recomputes the last one (its epilogue stores nothing)
       const int m = PAIR ? min(2 * (tile / p.n_tiles_n) + rank, m_tiles - 1) : tile / p.n_tiles_n;
@@ -225,7 +284,7 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
     // block, so everything that does not change is formed once: the operand descriptors differ
     // between stages only in their 14-bit address field (16-byte units; shared memory is far
     // below the field's range, so plain additions never carry out of it).
-    uint32_t stage = 0, phase = 0, acc_phase = 0;
+    uint32_t stage = 0, phase = 0, acc_phase = 0, a_stage = 0, a_phase = 0;
     int acc = 0;
     bool ok = true;
     const uint64_t a_desc0 = make_smem_desc(smem_u32(smem), SBO, LAYOUT);
@@ -237,7 +296,39 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
       if (!ok) break;
       tc_fence_after();   // the epilogue's TMEM reads of this buffer come before the MMAs that overwrite it
       const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BLOCK_N);
-      for (int it = 0; it < k_iters; ++it) {
+      if (HALO) {
+        // Output pixel (py, px) of the 8 x 16 patch reads halo pixel (py + ky, px + kx): the A operand
+        // of a tap is the same shared-memory patch, entered (ky * 16 + kx) pixel rows of 128 bytes
+        // further on.  The 8 pixels of one patch row are one 8-row operand group; groups are one halo
+        // row = 2048 bytes apart.  The 128-byte swizzle is a function of the shared-memory address
+        // (the TMA unit wrote the patch that way), so an operand that starts kx rows into a 1024-byte
+        // pattern needs nothing but its start address.
+        uint32_t first = 1;
+        for (int sg = 0; sg < slabs_per_tap && ok; ++sg) {
+          ok = mbar_wait(smem_u32(afull_bar + a_stage), a_phase, abort_flag, p.status, 0xA00 + (int)a_stage, wait_limit);
+          if (!ok) break;
+          const uint32_t a_base = smem_u32(smem_a + a_stage * Cfg::HALO_A_BYTES);
+#pragma unroll 1
+          for (int tap = 0; tap < 9; ++tap) {
+            ok = mbar_wait(full0 + 8u * stage, phase, abort_flag, p.status, 0x300 + (int)stage, wait_limit);
+            if (!ok) break;
+            const int ky = tap / 3, kx = tap - ky * 3;
+            const uint64_t a_tap = make_smem_desc(a_base + (uint32_t)((ky * Cfg::HALO_PITCH + kx) * 128), Cfg::HALO_PITCH * 128u, LAYOUT);
+            const uint64_t b_tap = a_desc;               // a_desc walks the weight ring in this mode
+            umma_bf16(d_tmem, a_tap, b_tap, IDESC, first ? 0u : 1u);
+            first = 0;
+#pragma unroll
+            for (int k = 1; k < SLAB_C / UMMA_K; ++k) umma_bf16(d_tmem, a_tap + (uint64_t)(2 * k), b_tap + (uint64_t)(2 * k), IDESC, 1u);
+            umma_commit(empty0 + 8u * stage);
+            a_desc += (uint64_t)(Cfg::B_BYTES >> 4);
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; a_desc = a_desc0; }
+          }
+          if (!ok) break;
+          umma_commit(smem_u32(aempty_bar + a_stage));   // the patch is free once all nine taps have read it
+          if (++a_stage == (uint32_t)A_STAGES) { a_stage = 0; a_phase ^= 1u; }
+        }
+      }
+      for (int it = 0; it < k_iters && !HALO; ++it) {
         // the copies complete on the barrier through the async proxy, which the MMAs read through too
         ok = mbar_wait(full0 + 8u * stage, phase, abort_flag, p.status, 0x300 + (int)stage, wait_limit);
         if (!ok) break;
@@ -271,7 +362,7 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
     const bool wide_out = EPI == TC_EPI_LSTM ? (p.hidden & 15) == 0 : (p.cout & 15) == 0;
     const int half = (warp - EPI_WARP0) >> 2;     // which half of the tile's columns
     const int row = quarter * 32 + lane;          // row of the 128-row tile = pixel of the patch
-    const int py = row / PATCH_W, px = row % PATCH_W;
+    const int py = row / PW, px = row % PW;
     uint32_t acc_phase = 0;
     int acc = 0;
     bool ok = true;
@@ -281,7 +372,7 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
       const int m_raw = PAIR ? 2 * (tile / p.n_tiles_n) + rank : tile / p.n_tiles_n;
       const int m = min(m_raw, m_tiles - 1);
       const int tx = m % p.tiles_x, ty = (m / p.tiles_x) % p.tiles_y, img = m / tiles_per_img;
-      const int x = tx * PATCH_W + px, y = ty * PATCH_H + py;
+      const int x = tx * PW + px, y = ty * PH + py;
       const bool valid = x < p.Wo && y < p.Ho && m_raw < m_tiles;
       const size_t pix = (size_t)y * p.Wo + x;
       const int col0 = nt * BLOCK_N + half * HALF_N;  // first packed output column of this warp
@@ -445,8 +536,26 @@ cudaError_t launch_pair(const ConvTcParams& p, int sm_count, cudaStream_t s) {
   return cudaLaunchKernelEx(&cfg, kern, p);
 }
 
+// Halo mode: one haloed activation patch per channel slab instead of one box per tap.
+template <int BLOCK_N, int EPI>
+cudaError_t launch_halo(const ConvTcParams& p, int sm_count, cudaStream_t s) {
+  using Cfg = TcCfg<BLOCK_N, 64>;
+  auto kern = conv_tc_kernel<BLOCK_N, 64, EPI, false, 1, true>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::HALO_SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  const int total_tiles = p.K * p.tiles_x * p.tiles_y * p.n_tiles_n;
+  const int grid = total_tiles < sm_count ? total_tiles : sm_count;
+  return launch_kernel(kern, grid, TC_THREADS, Cfg::HALO_SMEM_BYTES, s, p, p.pdl != 0);
+}
+
 template <int EPI>
 cudaError_t launch_shape(const ConvTcParams& p, int sm_count, cudaStream_t s) {
+  if (p.halo) {
+    if (EPI != TC_EPI_LSTM || p.slab_c != 64 || p.stride != 1 || p.pair) return cudaErrorInvalidValue;
+    if (p.block_n == 256) return launch_halo<256, TC_EPI_LSTM>(p, sm_count, s);
+    if (p.block_n == 128) return launch_halo<128, TC_EPI_LSTM>(p, sm_count, s);
+    return cudaErrorInvalidValue;
+  }
   if (p.pair) {
     if (p.slab_c == 64 && p.block_n == 256) return launch_pair<256, 64, EPI>(p, sm_count, s);
     return cudaErrorInvalidValue;

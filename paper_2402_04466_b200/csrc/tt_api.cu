@@ -41,6 +41,8 @@ struct TcLayer {
   float* b = nullptr;          // packed order
   int cin0 = 0, cin1 = 0, cout = 0, slab_c = 64, stride = 1;
   TensorMap128 maps_a[8];
+  TensorMap128 maps_halo[2];   // stride-1 layers of 64-channel slabs: haloed-patch boxes of the two sources
+  bool has_halo = false;
   TensorMap128 map_b[3];       // block_n = 64, 128, 256
   bool has_b[3] = {false, false, false};
 };
@@ -591,6 +593,18 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
                               ctx->Wm, ctx->Cx, 1, L.slab_c)) != TT_OK)
         return st;
       if ((st = make_act_maps(ctx, &L.maps_a[4], ctx->h_bf16, 2 * S, ctx->Hm, ctx->Wm, ctx->Ch, 1, L.slab_c)) != TT_OK) return st;
+      if (L.slab_c == 64 && !c.options[TT_OPT_NO_HALO]) {
+        // haloed patch of an 8 x 16 output tile: 18 rows of 16 pixels (10 are needed; the pitch keeps the swizzle phase)
+        const cuuint32_t box[4] = {64, 16, 18, 1};
+        struct { __nv_bfloat16* base; int n_img, C; } srcs[2] = {{reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[c.n_enc - 1]), S, ctx->Cx},
+                                                                {ctx->h_bf16, 2 * S, ctx->Ch}};
+        for (int i = 0; i < 2; ++i) {
+          const cuuint64_t dims[4] = {(cuuint64_t)srcs[i].C, (cuuint64_t)ctx->Wm, (cuuint64_t)ctx->Hm, (cuuint64_t)srcs[i].n_img};
+          const cuuint64_t str[3] = {(cuuint64_t)srcs[i].C * 2, (cuuint64_t)ctx->Wm * srcs[i].C * 2, (cuuint64_t)ctx->Hm * ctx->Wm * srcs[i].C * 2};
+          if ((st = encode_map(ctx, &L.maps_halo[i], srcs[i].base, 4, dims, str, box, 128)) != TT_OK) return st;
+        }
+        L.has_halo = true;
+      }
     } else if (no_post_tc || !post_tc_supported(ctx->Ch, (int)plane)) {
       return fail(ctx, TT_ERR_UNSUPPORTED, "a bf16 feed-forward model needs a last encoder width in multiples of 64 (at most 512) and "
                                            "a map of at least 128 pixels: its heads run on the tensor cores only");
@@ -752,6 +766,12 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
       q.pair = (bi == 2 && L.slab_c == 64 && L.has_b[1] && ctx->cta_pairs && K * q.tiles_x * q.tiles_y >= 2) ? 1 : 0;
       if (q.pair) q.map_b = L.map_b[1];
       q.two_per_sm = (encoder && ctx->enc_two_per_sm) ? 1 : 0;
+      if (!encoder && L.has_halo && !q.pair && (bi == 2 || bi == 1)) {
+        q.halo = 1;
+        q.maps_halo[0] = L.maps_halo[0];
+        q.maps_halo[1] = L.maps_halo[1];
+        q.tiles_x = (Wo + 7) / 8; q.tiles_y = (Ho + 15) / 16;
+      }
       q.cout = L.cout; q.bias = L.b; q.status = ctx->status_dev; q.wait_limit = ctx->wait_limit;
       q.n_prod = 3;
       q.pdl = ctx->profiling ? 0 : 1;

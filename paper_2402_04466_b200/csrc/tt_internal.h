@@ -114,6 +114,7 @@ struct ConvTcParams {
   // A operand sources: up to two NHWC bf16 tensors (x then h); for stride 2 four parity
   // views of the single source.  maps_a[src*4 + parity] with parity = (ypar*2 + xpar).
   TensorMap128 maps_a[8];
+  TensorMap128 maps_halo[2];// halo mode: the two sources again with a box of [64 channels][16][18][1] (haloed patch of an 8 x 16 tile)
   TensorMap128 map_b;       // packed weights [CoutPacked][Ktot] bf16, K-major
   int32_t n_src;            // 1 or 2
   int32_t slabs[2];         // channel slabs (of slab_c channels) per source
@@ -127,6 +128,7 @@ struct ConvTcParams {
   int32_t block_n;          // 64, 128 or 256
   int32_t n_prod;           // producer warps that issue loads, 1..3
   int32_t two_per_sm;       // encoder layers with tiles up to 128 wide: two blocks per multiprocessor, half the ring each
+  int32_t halo;             // stride-1 layer of 64-channel slabs: one haloed patch per channel slab, 8 x 16 output patches
   int32_t pair;             // run as CTA pairs (cta_group::2): block_n 256, map_b's box then holds 128 rows
   int32_t pdl;              // launch as a programmatic dependent of the previous kernel in the stream
   int32_t cout;             // real output channels (RELU) or 4*hidden (LSTM)

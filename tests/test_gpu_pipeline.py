@@ -13,10 +13,10 @@ from parity_util import assert_close, check_masks, check_reductions_from_own_mas
 pytestmark = pytest.mark.gpu
 
 
-def _make(wl, K=1, overlay=None, precision=None, timeout_ns=0, plain_launches=False, cta_pairs=False):
+def _make(wl, K=1, overlay=None, precision=None, timeout_ns=0, plain_launches=False, cta_pairs=False, halo=True):
     weights = tt_synth.make_weights(wl)
     cfg = binding.make_config(wl, max_streams=K, overlay=overlay, precision=precision, sync_timeout_ns=timeout_ns,
-                              plain_launches=plain_launches, cta_pairs=cta_pairs)
+                              plain_launches=plain_launches, cta_pairs=cta_pairs, halo=halo)
     ctx = binding.Context(cfg, weights)
     states = [ctx.state_create() for _ in range(K)]
     return ctx, states, weights
@@ -228,7 +228,8 @@ def test_bf16_wide_channels_small_map(cuda_device):
 def test_bf16_cta_pairs_with_an_odd_number_of_tiles(cuda_device):
     """On request the 256-wide ConvLSTM tiles run on CTA pairs (two neighbouring 128-pixel tiles per MMA).  Three
     streams of an 80x40 map give 75 tiles: the last pair has no second tile, its second CTA recomputes the last
-    tile and must store nothing.  Checked against the oracle, and bit for bit against the default single-CTA tiles."""
+    tile and must store nothing.  Checked against the oracle, and bit for bit against single-CTA tiles that add up
+    the taps in the same order (one activation box per tap)."""
     wl = tt_synth.workload("cfg1-gain").with_(name="bf16-pairs", src_w=854, src_h=320, net_w=640, net_h=320)
     assert wl.map_hw() == (40, 80)
     _run_bf16(cuda_device, wl, 3, 2, cta_pairs=True)
@@ -236,7 +237,7 @@ def test_bf16_cta_pairs_with_an_odd_number_of_tiles(cuda_device):
     frames = _frames(wl, K, n)
     outs = []
     for pairs in (True, False):
-        ctx, states, _ = _make(wl, K, cta_pairs=pairs)
+        ctx, states, _ = _make(wl, K, cta_pairs=pairs, halo=False)
         for t in range(n):
             ctx.submit_frames([torch.from_numpy(frames[k][t]).to(cuda_device) for k in range(K)], states, frame_index=t)
             res = ctx.sync()
@@ -276,6 +277,31 @@ def test_bf16_postprocess_from_the_fp32_state_still_matches(cuda_device):
             assert_close(got[0][k][1], got[1][k][1], 2 * TOL_OUT, "confidences of the two postprocess kernels")
     for ctx, _ in ctxs:
         ctx.destroy()
+
+
+def test_bf16_convlstm_one_box_per_tap_still_matches(cuda_device):
+    """By default the ConvLSTM fetches one haloed activation patch per channel slab and reads all nine taps from it
+    (every other bf16 test runs that way).  The form with one activation box per tap stays available; both must
+    match the oracle, and each other up to the order in which the fp32 accumulator adds the taps up."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="tapbox", src_w=214, src_h=120, net_w=176, net_h=136, hidden=64)
+    K, n = 2, 3
+    frames = _frames(wl, K, n)
+    outs = []
+    for halo in (True, False):
+        ctx, states, w = _make(wl, K, halo=halo)
+        oras = [oracle.OraclePipeline(wl, w) for _ in range(K)]
+        for t in range(n):
+            ctx.submit_frames([torch.from_numpy(frames[k][t]).to(cuda_device) for k in range(K)], states, frame_index=t)
+            res = ctx.sync()
+            for k in range(K):
+                ref = oras[k].step(frames[k][t], want_overlay=False)
+                band = max(1e-3, BAND_REL * float(np.sqrt(np.mean(ref.z.astype(np.float64) ** 2))))
+                _compare_frame(ctx, states[k], res[k], ref, TOL_OUT, band, tag=f"tapbox halo={halo} k={k} t={t}", tol_mid=TOL_MID_PLAIN,
+                               max_band_frac=MAX_BAND_FRAC)
+        outs.append([ctx.debug_tensor(s, "c") for s in states])
+        ctx.destroy()
+    for a, b in zip(*outs):
+        assert rms_err(a, b) < 1e-3
 
 
 def test_bf16_stride1_encoder_and_overlay(cuda_device):
