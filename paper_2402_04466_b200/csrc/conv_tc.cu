@@ -64,10 +64,11 @@ struct TcCfg {
   // columns are needed; a row pitch of 16 pixels = 2048 bytes keeps every 8-pixel operand group
   // of every tap at the same phase of the 1024-byte swizzle pattern).  The weight ring holds one
   // [BLOCK_N][64] slab per tap.
-  static constexpr int HALO_PITCH = 16, HALO_ROWS = 18;
-  static constexpr int HALO_A_BYTES = HALO_ROWS * HALO_PITCH * SLAB_C * 2;   // 36864
+  static constexpr int HALO_PITCH = 10, HALO_ROWS = 18;
+  static constexpr int HALO_A_BYTES = (HALO_ROWS * HALO_PITCH * SLAB_C * 2 + 1023) / 1024 * 1024;   // 23040 -> 23552
+  static constexpr int HALO_A_TX = HALO_ROWS * HALO_PITCH * SLAB_C * 2;
   static constexpr int HALO_A_STAGES = 2;
-  static constexpr int HALO_B_RAW = (204 * 1024 - HALO_A_STAGES * HALO_A_BYTES) / B_BYTES;
+  static constexpr int HALO_B_RAW = (210 * 1024 - HALO_A_STAGES * HALO_A_BYTES) / B_BYTES;
   static constexpr int HALO_B_STAGES = HALO_B_RAW > 8 ? 8 : HALO_B_RAW;
   static constexpr int HALO_SMEM_BYTES = HALO_B_STAGES * B_BYTES + HALO_A_STAGES * HALO_A_BYTES + BAR_BYTES + TAB_BYTES + 1024;
   static_assert(STAGES >= N_PROD, "every producer needs a stage of its own");
@@ -230,7 +231,7 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
             if (!ok) break;
             const int src = sg < p.slabs[0] ? 0 : 1;
             const uint32_t ab = smem_u32(afull_bar + a_stage);
-            mbar_arrive_expect_tx(ab, Cfg::HALO_A_BYTES);
+            mbar_arrive_expect_tx(ab, Cfg::HALO_A_TX);
             tma_load_4d(smem_u32(smem_a + a_stage * Cfg::HALO_A_BYTES), &p.maps_halo[src], ab, (src ? sg - p.slabs[0] : sg) * SLAB_C,
                         tx * PW - 1, ty * PH - 1, src ? img_h : img_x);
           }

@@ -595,7 +595,7 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
       if ((st = make_act_maps(ctx, &L.maps_a[4], ctx->h_bf16, 2 * S, ctx->Hm, ctx->Wm, ctx->Ch, 1, L.slab_c)) != TT_OK) return st;
       if (L.slab_c == 64 && !c.options[TT_OPT_NO_HALO]) {
         // haloed patch of an 8 x 16 output tile: 18 rows of 16 pixels (10 are needed; the pitch keeps the swizzle phase)
-        const cuuint32_t box[4] = {64, 16, 18, 1};
+        const cuuint32_t box[4] = {64, 10, 18, 1};
         struct { __nv_bfloat16* base; int n_img, C; } srcs[2] = {{reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[c.n_enc - 1]), S, ctx->Cx},
                                                                 {ctx->h_bf16, 2 * S, ctx->Ch}};
         for (int i = 0; i < 2; ++i) {
