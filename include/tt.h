@@ -333,7 +333,10 @@ tt_status tt_preprocess(const uint8_t* src_dev, int32_t K, int64_t src_frame_str
  * scratch_dev: tt_postprocess_scratch_bytes(...) bytes of device memory, 8-byte aligned; the call
  * clears it first, contents on entry are ignored.
  * hidden must be a multiple of 4 and at most 512; hm, wm at most 16384.  A misaligned or null
- * pointer is answered with TT_ERR_INVALID_ARG before anything is launched.
+ * pointer is answered with TT_ERR_INVALID_ARG before anything is launched.  The stage-level calls
+ * have no status word: a bounded device-side wait that ran out inside them (which no healthy
+ * device produces) leaves the outputs incomplete without an error code; contexts report it
+ * through tt_sync.
  */
 size_t tt_postprocess_scratch_bytes(int32_t K, int32_t hm, int32_t wm, int32_t hidden, int32_t n_tools);
 tt_status tt_postprocess(const float* h_dev, int32_t channels_last, int32_t K, int32_t hm, int32_t wm,
