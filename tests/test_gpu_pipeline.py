@@ -304,6 +304,14 @@ def test_bf16_convlstm_one_box_per_tap_still_matches(cuda_device):
         assert rms_err(a, b) < 1e-3
 
 
+def test_bf16_eight_tools_and_mean_sigmoid_confidence(cuda_device):
+    """The tensor-core heads with every tool slot in use and the confidence taken as the mean probability (the
+    fixed-point probability sums instead of the confidence-head columns)."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="bf16-t8", src_w=214, src_h=120, net_w=176, net_h=136, hidden=64, n_tools=8,
+                                              conf_mode="mean_sigmoid")
+    _run_bf16(cuda_device, wl, 3, 2)
+
+
 def test_bf16_stride1_encoder_and_overlay(cuda_device):
     wl = tt_synth.workload("cfg1-gain").with_(name="bf16-s1", src_w=96, src_h=72, net_w=64, net_h=48,
                                               enc_cout=(32, 64), enc_stride=(2, 1), hidden=32, overlay=True)
