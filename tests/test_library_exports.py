@@ -86,3 +86,14 @@ def test_stage_level_calls_refuse_misaligned_or_oversized_arguments_on_the_host(
     assert lib.tt_debug_expire_wait(None, 1000) == 1
     assert lib.tt_render_layers(A, 1, 0, 8, 8, 24, A + 0x10000, 4, 4, 4, pal, 0, 0, A + 0x20000, None) == 1      # layers < 1
     assert lib.tt_render_layers(A, 1, 0, 8, 8, 24, A + 0x10000, 4, 4, 4, pal, 2, 0, A + 0x20001, None) == 1      # misaligned output
+
+
+def test_option_indices_in_the_binding_match_the_header():
+    text = open(os.path.join(ROOT, "include", "tt.h")).read()
+    declared = {name: int(val) for name, val in re.findall(r"\b(TT_OPT_[A-Z_0-9]+)\s*=\s*(\d+)", text)}
+    assert declared and len(set(declared.values())) == len(declared) and max(declared.values()) < 8
+    for name, val in declared.items():
+        assert getattr(binding, name) == val, name
+    for name in dir(binding):
+        if name.startswith("TT_OPT_"):
+            assert name in declared, f"{name} is not in tt.h"
