@@ -102,8 +102,8 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 // Tile loads of a CTA pair: data lands in the issuing CTA's shared memory, the transaction bytes
-// are counted on the barrier given by its cluster address (the leader's).  No multicast: every CTA
-// fetches its own tiles.
+// are counted on the barrier given by its cluster address (the leader's).  Every CTA fetches its
+// own tiles; nothing is broadcast.
 __device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const void* tmap, uint32_t cluster_bar, int c0, int c1,
                                                  int c2, int c3) {
   asm volatile(
@@ -127,10 +127,11 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc,
       : "memory");
 }
 // arrives, once the pair's MMAs issued so far are complete, on the barrier at the same
-// shared-memory offset in both CTAs of the pair
+// shared-memory offset in both CTAs of the pair: one commit per CTA, the peer's barrier addressed
+// through its cluster address
 __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-               ::"r"(bar), "h"((uint16_t)3) : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(map_to_cta(bar, 1u)) : "memory");
 }
 
 // Named barrier over `count` threads that also ORs a flag across them: every participant learns
