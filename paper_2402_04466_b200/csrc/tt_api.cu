@@ -140,11 +140,11 @@ struct tt_ctx {
   int q_head = 0, q_count = 0;      // oldest in-flight slot, number in flight
   int bound = 0;                    // slot whose resources the view members hold
   int last_done = -1;               // slot of the last completed submit (debug taps)
-  // CUDA graphs of the tick's launch sequence, one per (stream count, slot, state placement).  Frame
-  // pointers change every tick, so the kernels read them from a small device table per slot that
-  // is refreshed by a 64-byte copy in front of the graph launch.
+  // CUDA graphs of the tick's launch sequence, one per (stream count, slot, pointer table, state placement).
+  // Frame pointers may change every tick, so the kernels read them from a small device table; a table that
+  // does not yet hold the tick's pointers is refreshed by a 64-byte copy in front of the graph launch.
   struct TickGraph {
-    int K = 0, slot = 0, flat = 0;
+    int K = 0, slot = 0, flat = 0, tab = 0;
     int sig[TT_MAX_STREAMS] = {};   // state slot * 2 + half of every batch position
     int seen = 0;                   // direct executions of this key so far (capture happens on the second)
     uint64_t launches = 0;          // kernels inside the graph
@@ -155,8 +155,15 @@ struct tt_ctx {
   bool cta_pairs = false;           // TT_OPT_CTA_PAIRS
   bool enc_two_per_sm = true;       // !TT_OPT_ENC_ONE_PER_SM
   bool feed_forward = false;        // TT_OPT_FEED_FORWARD: no recurrent cell, the heads read the encoder output
-  const uint8_t** frame_tab_dev[2] = {nullptr, nullptr};   // device, [TT_MAX_STREAMS] pointers per slot
-  const uint8_t** frame_tab_host[2] = {nullptr, nullptr};  // pinned staging of the same
+  // Every slot owns a few device tables, each remembering the set of frame pointers it holds: a caller whose
+  // frames arrive in a fixed set of buffers (a capture ring; the slot's own staging buffer for host frames) finds
+  // its pointers already on the device and no copy is enqueued.
+  static constexpr int FRAME_TABS = 4;
+  const uint8_t** frame_tab_dev[2] = {nullptr, nullptr};   // device, [FRAME_TABS][TT_MAX_STREAMS] pointers per slot
+  const uint8_t** frame_tab_host[2] = {nullptr, nullptr};  // pinned staging of one table
+  const uint8_t* frame_tab_last[2][FRAME_TABS][TT_MAX_STREAMS] = {};   // what each device table holds
+  bool frame_tab_valid[2][FRAME_TABS] = {};
+  uint64_t frame_tab_used[2][FRAME_TABS] = {};             // tick at which the table was last used (the oldest is replaced)
   const uint8_t* const* cur_tab = nullptr;                  // table the tick being enqueued reads
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_copy = nullptr;
@@ -505,7 +512,7 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
     *sl.status_host = 0;
     {
       uint64_t* tab = nullptr;
-      if ((st = dev_alloc(ctx, &tab, (size_t)TT_MAX_STREAMS)) != TT_OK) return st;
+      if ((st = dev_alloc(ctx, &tab, (size_t)tt_ctx::FRAME_TABS * TT_MAX_STREAMS)) != TT_OK) return st;
       ctx->frame_tab_dev[i] = reinterpret_cast<const uint8_t**>(tab);
       TT_CUDA(ctx, cudaHostAlloc(reinterpret_cast<void**>(&ctx->frame_tab_host[i]), sizeof(void*) * TT_MAX_STREAMS, cudaHostAllocDefault));
     }
@@ -1013,36 +1020,55 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
     TT_CUDA(ctx, cudaEventRecord(ctx->ev_copy, ctx->copy_stream));
     TT_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_copy, 0));
   }
-  // frame pointers of this tick -> the slot's device table (the kernels read them from there)
-  for (int n = 0; n < TT_MAX_STREAMS; ++n) ctx->frame_tab_host[slot][n] = n < K ? fp.p[n] : nullptr;
-  TT_CUDA(ctx, cudaMemcpyAsync(ctx->frame_tab_dev[slot], ctx->frame_tab_host[slot], sizeof(void*) * TT_MAX_STREAMS,
-                               cudaMemcpyHostToDevice, s));
-  ctx->cur_tab = ctx->frame_tab_dev[slot];
+  // frame pointers of this tick -> the slot's device table (the kernels read them from there).  The copy is
+  // skipped when the table already holds these pointers: always the case for host frames (they are staged in
+  // the slot's own buffer) and for callers whose frames arrive in a fixed set of device buffers.
+  int tab = -1, oldest = 0;
+  for (int i = 0; i < tt_ctx::FRAME_TABS && tab < 0; ++i) {
+    bool same = ctx->frame_tab_valid[slot][i];
+    for (int n = 0; n < TT_MAX_STREAMS && same; ++n) same = ctx->frame_tab_last[slot][i][n] == (n < K ? fp.p[n] : nullptr);
+    if (same) tab = i;
+    if (ctx->frame_tab_used[slot][i] < ctx->frame_tab_used[slot][oldest]) oldest = i;
+  }
+  if (tab < 0) {
+    tab = oldest;
+    for (int n = 0; n < TT_MAX_STREAMS; ++n) ctx->frame_tab_last[slot][tab][n] = ctx->frame_tab_host[slot][n] = n < K ? fp.p[n] : nullptr;
+    ctx->frame_tab_valid[slot][tab] = false;   // stays so if the copy cannot be enqueued
+    TT_CUDA(ctx, cudaMemcpyAsync(ctx->frame_tab_dev[slot] + tab * TT_MAX_STREAMS, ctx->frame_tab_host[slot],
+                                 sizeof(void*) * TT_MAX_STREAMS, cudaMemcpyHostToDevice, s));
+    ctx->frame_tab_valid[slot][tab] = true;
+  }
+  ctx->frame_tab_used[slot][tab] = ctx->n_ticks + 1;
+  ctx->cur_tab = ctx->frame_tab_dev[slot] + tab * TT_MAX_STREAMS;
   // everything that moves host data to the device (frames, pointer table) counts as the H2D stage
   st = mark_stage(ctx, TT_STAGE_H2D, 0);
   if (st != TT_OK) return st;
 
-  // The launch sequence of a tick is replayed from a CUDA graph once the same (K, slot, state
-  // placement) has been seen before; the first occurrence runs as plain launches.  With stage
-  // events requested the tick always runs as plain launches.
+  // The launch sequence of a tick is replayed from a CUDA graph.  Which kernel variants a tick launches depends
+  // on the stream count and the frames' alignment alone, so the first tick of such a family runs as plain
+  // launches (modules load, attributes are set outside any capture); after it, every new (slot, pointer
+  // table, state placement) of the family is captured the first time it shows up.  With stage events
+  // requested the tick always runs as plain launches.
   tt_ctx::TickGraph* tg = nullptr;
+  bool family_warm = false;
   if (!ctx->graphs_off && !ctx->profiling) {
     int flat = 1;
     // the overlay launch picks its word-wise variant from the frames' 4-byte alignment: part of the key
     for (int n = 0; n < K; ++n) flat &= (((uintptr_t)fp.p[n] & 3) == 0) ? 1 : 0;
     for (auto& g : ctx->graphs) {
-      bool same = g.K == K && g.slot == slot && g.flat == flat;
+      family_warm |= g.K == K && g.flat == flat && (g.seen >= 1 || g.exec);
+      bool same = g.K == K && g.slot == slot && g.flat == flat && g.tab == tab;
       for (int n = 0; n < K && same; ++n) same = g.sig[n] == states[n]->slot * 2 + states[n]->half;
       if (same) { tg = &g; break; }
     }
     if (!tg) {
-      if (ctx->graphs.size() >= 64) {            // bounded cache: drop everything and start over
+      if (ctx->graphs.size() >= 128) {            // bounded cache: drop everything and start over
         for (auto& g : ctx->graphs)
           if (g.exec) cudaGraphExecDestroy(g.exec);
         ctx->graphs.clear();
       }
       tt_ctx::TickGraph g;
-      g.K = K; g.slot = slot; g.flat = flat;
+      g.K = K; g.slot = slot; g.flat = flat; g.tab = tab;
       for (int n = 0; n < K; ++n) g.sig[n] = states[n]->slot * 2 + states[n]->half;
       ctx->graphs.push_back(g);
       tg = &ctx->graphs.back();
@@ -1052,8 +1078,8 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
     TT_CUDA(ctx, cudaGraphLaunch(tg->exec, s));
     ctx->n_launches += tg->launches;
     ctx->n_ticks += 1;
-  } else if (tg && tg->seen >= 1) {
-    // second occurrence: capture the sequence (kernels plus the two result copies), then launch it
+  } else if (tg && (tg->seen >= 1 || family_warm)) {
+    // capture the sequence (kernels plus the two result copies), then launch it
     const uint64_t launches_before = ctx->n_launches;
     cudaGraph_t graph = nullptr;
     cudaError_t ce = cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal);

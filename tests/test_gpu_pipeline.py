@@ -461,6 +461,40 @@ def test_graph_replay_matches_plain_launches(cuda_device):
         assert np.array_equal(h1, h2) and np.array_equal(c1, c2)
 
 
+def test_frames_in_a_ring_of_device_buffers_of_any_length(cuda_device):
+    """The context remembers which frame pointers its device-side pointer tables hold and skips the table
+    refresh when a tick brings a known set.  Frames delivered through rings of 1, 3 and 10 buffer sets (always
+    known; known after one round; more sets than tables, so the oldest is replaced every tick) must give
+    the same bits as kernel-by-kernel launches from the same rings."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="ring", src_w=214, src_h=120, net_w=160, net_h=120, overlay=True)
+    K, n = 2, 13
+    host = _frames(wl, K, n)
+    runs = {}
+    for ring, plain in ((1, True), (1, False), (3, False), (10, False), (10, True)):
+        bufs = [[torch.empty_like(torch.from_numpy(host[k][0]), device=cuda_device) for _ in range(ring)] for k in range(K)]
+        ctx, states, _ = _make(wl, K, overlay=True, plain_launches=plain)
+        out = []
+        for t in range(n):
+            who = (0, 1) if t % 5 != 4 else (1,)        # the batch shrinks now and then: a different pointer set
+            for k in who:
+                bufs[k][t % ring].copy_(torch.from_numpy(host[k][t]))
+            ctx.submit_frames([bufs[k][t % ring] for k in who], [states[k] for k in who], frame_index=t)
+            out.append([(x["frame_index"], ctx.fetch_probs(x), ctx.fetch_overlay(x), x["conf"].copy(), x["cx"].copy())
+                        for x in ctx.sync()])
+        runs[(ring, plain)] = (out, [ctx.state_export(s) for s in states])
+        ctx.destroy()
+    ref_out, ref_h = runs[(1, True)]
+    for key, (out, hs) in runs.items():
+        for ra, rb in zip(ref_out, out):
+            assert len(ra) == len(rb)
+            for xa, xb in zip(ra, rb):
+                assert xa[0] == xb[0]
+                for va, vb in zip(xa[1:], xb[1:]):
+                    assert np.array_equal(va, vb), key
+        for (h1, c1), (h2, c2) in zip(ref_h, hs):
+            assert np.array_equal(h1, h2) and np.array_equal(c1, c2), key
+
+
 def test_dependent_launches_change_no_bit(cuda_device):
     """The tensor-core kernels normally start as programmatic dependents of their predecessor (set-up overlapping
     its tail); with stage profiling on every kernel is launched normally behind an event.  Both must give the same
