@@ -48,7 +48,7 @@ def load_peaks():
 
 
 KERNEL_SOURCES = {"convlstm": ["conv_tc.cu", "tc_ptx.cuh"], "enc1": ["conv_tc.cu", "tc_ptx.cuh"], "enc2": ["conv_tc.cu", "tc_ptx.cuh"],
-                  "enc0": ["conv_first_tc.cu", "tc_ptx.cuh"], "preprocess": ["preprocess.cu"], "postprocess": ["post_tc.cu", "tc_ptx.cuh"],
+                  "enc0": ["conv_first_tc.cu", "tc_ptx.cuh", "pre_math.cuh"], "preprocess": ["preprocess.cu", "pre_math.cuh"], "postprocess": ["post_tc.cu", "tc_ptx.cuh"],
                   "overlay": ["overlay.cu"]}
 
 

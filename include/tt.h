@@ -65,6 +65,9 @@ typedef enum {
                                 (for A/B measurements) */
   TT_OPT_NO_HALO = 6,        /* ConvLSTM fetches one activation box per tap instead of one haloed patch per channel
                                 slab (for A/B measurements) */
+  TT_OPT_FUSED_PRE = 7,      /* bf16 path: run the preprocessing inside the first encoder layer instead of as a kernel of its
+                                own that writes the resized fp32 image (same bits; slower as measured, kept for A/B
+                                measurements; ignored where the layer or the resize factor does not allow it) */
   TT_OPT_NO_POST_TC = 3      /* bf16 path: post-process from the fp32 hidden state, not from its bf16 copy on the
                                 tensor cores (for A/B measurements; not available for feed-forward models) */
 } tt_option;

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "TT_OK", 1: "TT_ERR_INVALID_ARG", 2: "TT_ERR_UNSUPPORTED", 3:
                 5: "TT_ERR_ADMISSION", 6: "TT_ERR_NOT_READY", 7: "TT_ERR_TIMEOUT", 8: "TT_ERR_DEVICE_STATUS"}
 TT_FP32, TT_BF16 = 0, 1
 TT_OPT_PLAIN_LAUNCHES, TT_OPT_FEED_FORWARD, TT_OPT_CTA_PAIRS, TT_OPT_NO_POST_TC, TT_OPT_RESERVED_SMS = 0, 1, 2, 3, 4
-TT_OPT_ENC_ONE_PER_SM, TT_OPT_NO_HALO = 5, 6
+TT_OPT_ENC_ONE_PER_SM, TT_OPT_NO_HALO, TT_OPT_FUSED_PRE = 5, 6, 7
 TT_CONF_MEAN_SIGMOID, TT_CONF_GAP_LINEAR = 0, 1
 TENSOR_IDS = {"pre": 0, "enc0": 1, "enc1": 2, "enc2": 3, "enc3": 4, "h": 8, "c": 9, "logits": 10, "prob": 11}
 
@@ -153,10 +153,12 @@ def _check(lib, status: int, ctx=None):
 def make_config(wl, max_streams: int = 1, device: int = 0, overlay: Optional[bool] = None,
                 cuda_stream: int = 0, sync_timeout_ns: int = 0, precision: Optional[str] = None,
                 plain_launches: bool = False, cta_pairs: bool = False, post_tc: bool = True,
-                reserved_sms: int = 0, enc_two_per_sm: bool = True, halo: bool = True) -> tt_config:
+                reserved_sms: int = 0, enc_two_per_sm: bool = True, halo: bool = True,
+                fused_pre: bool = False) -> tt_config:
     """Fill a tt_config from any object carrying the workload attributes (src_w, net_w, enc_cout, ...).
 
-    plain_launches=True makes every tick launch its kernels one by one instead of replaying a CUDA graph."""
+    plain_launches=True makes every tick launch its kernels one by one instead of replaying a CUDA graph.
+    fused_pre=True runs the preprocessing inside the first encoder layer (bf16 path; same bits, measured slower)."""
     cfg = tt_config()
     cfg.struct_size = C.sizeof(tt_config)
     cfg.abi_version = TT_ABI_VERSION
@@ -187,6 +189,7 @@ def make_config(wl, max_streams: int = 1, device: int = 0, overlay: Optional[boo
     cfg.options[TT_OPT_RESERVED_SMS] = reserved_sms
     cfg.options[TT_OPT_ENC_ONE_PER_SM] = 0 if enc_two_per_sm else 1
     cfg.options[TT_OPT_NO_HALO] = 0 if halo else 1
+    cfg.options[TT_OPT_FUSED_PRE] = 1 if fused_pre else 0
     return cfg
 
 

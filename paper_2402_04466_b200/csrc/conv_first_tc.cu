@@ -17,8 +17,16 @@
 // TMA tile store (full 128-byte lines to L2 instead of 16-byte pieces per thread; the part of a
 // border tile outside the image is clipped by the TMA unit).  The operand ring has 3 stages and the accumulator 2 buffers, so gather, MMA and
 // epilogue of different tiles overlap.  All waits are bounded (see tc_ptx.cuh).
+//
+// FUSED form: the preprocessing stage runs inside this kernel, and the resized fp32 image is never written to
+// or read from memory.  Four more warps build the patch instead of the TMA unit: bilinear resize +
+// normalisation with the expressions of the stand-alone preprocess kernel, so the fp32 values are the same bits.
+// They sample from frame rows staged in shared memory (rows are a byte stream: the 16-byte aligned range that
+// covers a row's part is staged); the rows of the tile two ahead travel through the same threads' registers
+// (128-bit loads issued before a tile is sampled, stored after it), so the memory latency hides behind the sampling.
 #include "tt_internal.h"
 #include "tc_ptx.cuh"
+#include "pre_math.cuh"
 
 namespace tt {
 namespace {
@@ -28,15 +36,45 @@ using namespace tc;
 constexpr int F_STAGES = 3;
 constexpr int F_A_BYTES = 128 * 64;                 // 128 rows x 32 bf16
 constexpr int F_THREADS = 288;                      // warps 0-3 gather, 4 MMA, 5-8 epilogue
+constexpr int F_THREADS_FUSED = F_THREADS + 128;    // warps 9-12 stage frame rows and sample them into the patch buffers
+constexpr int F_SRC_STAGES = 3;
+constexpr int F_SRC_PASSES = 4;                     // a staging pass moves 8 rows of up to 16 vectors: at most 32 rows of 256 bytes
+constexpr int F_SRC_BUDGET = 48 * 1024;             // shared memory the staged frame rows may take
+constexpr int F_MAX_TILES = 128;                    // tile columns and tile rows the fused form keeps source ranges for
 constexpr int F_TMEM_COLS = 128;                    // two accumulator buffers of up to 64 columns
 
 // Columns of the input patch box: 3 columns in front for alignment, the 15*stride + 3 columns of
 // the patch, rounded up to a multiple of 4 (16 bytes).
 __host__ __device__ constexpr int box_w(int stride) { return (15 * stride + 3 + 3 + 3) & ~3; }
 
-template <int COUT, int STRIDE>
-__global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
+// Six bytes starting at byte offset `b` of a word-aligned shared buffer: the RGB triples of two
+// neighbouring pixels.  lo = bytes b..b+3 (R0 G0 B0 R1), hi = bytes b+4..b+7 (G1 B1 . .).
+__device__ __forceinline__ void fetch_pair(const uint32_t* s_words, int b, uint32_t& lo, uint32_t& hi) {
+  const int w = b >> 2;
+  const uint32_t sh = (uint32_t)(b & 3) * 8u;
+  const uint32_t w0 = s_words[w], w1 = s_words[w + 1], w2 = s_words[w + 2];
+  lo = __funnelshift_r(w0, w1, sh);
+  hi = __funnelshift_r(w1, w2, sh);
+}
+
+struct TileAt {
+  int tx, ty, img;
+};
+// tile index -> (tile column, tile row, image) without integer divisions
+__device__ __forceinline__ TileAt tile_at(int tile, int tiles_x, int tiles_per_img, float inv_tiles_x, float inv_tiles_per_img) {
+  TileAt t;
+  t.img = pre::div_by(tile, tiles_per_img, inv_tiles_per_img);
+  const int rem = tile - t.img * tiles_per_img;
+  t.ty = pre::div_by(rem, tiles_x, inv_tiles_x);
+  t.tx = rem - t.ty * tiles_x;
+  return t;
+}
+
+template <int COUT, int STRIDE, bool FUSED>
+__global__ void __launch_bounds__(FUSED ? F_THREADS_FUSED : F_THREADS, FUSED ? 2 : 3)
+conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
   constexpr int PH = 7 * STRIDE + 3;                         // rows of the input patch of a 16 x 8 output tile
+  constexpr int PW = 15 * STRIDE + 3;                        // its columns
   constexpr int BW = box_w(STRIDE);                          // box columns: 3 alignment columns + the patch, rounded up to 4
   constexpr int PATCH_BYTES = 3 * PH * BW * 4;
   constexpr int PATCH_STRIDE = (PATCH_BYTES + 127) & ~127;   // patch buffers stay 128-byte aligned
@@ -45,14 +83,20 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
   uint8_t* s_a = s_out + 128 * COUT * 2;                      // operand ring
   uint8_t* s_b = s_a + F_STAGES * F_A_BYTES;                  // weights in operand layout
   uint8_t* s_patch = s_b + COUT * 64;                         // [2] patches of [3][PH][BW] floats
-  __shared__ __align__(8) uint64_t s_bar[2 * F_STAGES + 6];
+  uint8_t* s_src = s_patch + 2 * PATCH_STRIDE;                // FUSED: [F_SRC_STAGES] x src_rows_cap rows of src_row_cap bytes
+  __shared__ __align__(8) uint64_t s_bar[2 * F_STAGES + 8];
+  __shared__ const uint8_t* s_frame[TT_MAX_STREAMS];          // the batch's frame pointers
+  __shared__ int s_yoff0[2][PH], s_yoff1[2][PH];              // per patch row: byte offsets of its two source rows' first staged column, -1 outside
+  __shared__ float s_fy[2][PH];
+  __shared__ int s_gx[F_MAX_TILES][2], s_gy[F_MAX_TILES][2];  // first and last source column / row under every tile column / row
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   uint64_t* a_full = s_bar;                 // [F_STAGES] 128 gather threads arrive
   uint64_t* a_empty = s_bar + F_STAGES;     // [F_STAGES] MMA commit
   uint64_t* t_full = s_bar + 2 * F_STAGES;  // [2] MMA commit
   uint64_t* t_empty = t_full + 2;           // [2] 4 epilogue warps arrive
-  uint64_t* p_full = t_empty + 2;           // [2] patch landed (TMA transaction bytes)
+  uint64_t* p_full = t_empty + 2;           // [2] patch landed (TMA transaction bytes; FUSED: 128 sampling threads arrive)
+  uint64_t* p_empty = p_full + 2;           // [2] FUSED only: 128 gather threads have read the patch
   volatile int* abort_flag = &s_abort;
 
   pdl_launch_dependents();
@@ -66,7 +110,8 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(t_full + a), 1);
       mbar_init(smem_u32(t_empty + a), 4);
-      mbar_init(smem_u32(p_full + a), 1);
+      mbar_init(smem_u32(p_full + a), FUSED ? 128 : 1);
+      mbar_init(smem_u32(p_empty + a), 128);
     }
     s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -74,6 +119,22 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
   // weights: already packed in the operand layout, COUT * 64 bytes
   for (int i = threadIdx.x; i < COUT * 4; i += F_THREADS)
     reinterpret_cast<uint4*>(s_b)[i] = __ldg(reinterpret_cast<const uint4*>(p.w_packed) + i);
+  if (FUSED) {
+    if (threadIdx.x < TT_MAX_STREAMS) s_frame[threadIdx.x] = threadIdx.x < p.K ? (p.src_tab ? p.src_tab[threadIdx.x] : p.src.p[threadIdx.x]) : nullptr;
+    // the source pixels under the part of every tile column's / tile row's patch that lies inside the resized image
+    for (int i = threadIdx.x; i < p.tiles_x + p.tiles_y; i += F_THREADS_FUSED) {
+      if (i < p.tiles_x) {
+        const int first = max(i * 16 * STRIDE - 1, 0), last = min(i * 16 * STRIDE - 1 + PW - 1, p.W - 1);
+        s_gx[i][0] = pre::axis_sample(first, p.src_w, p.W).i0;
+        s_gx[i][1] = min(pre::axis_sample(last, p.src_w, p.W).i0 + 1, p.src_w - 1);
+      } else {
+        const int t = i - p.tiles_x;
+        const int first = max(t * 8 * STRIDE - 1, 0), last = min(t * 8 * STRIDE - 1 + PH - 1, p.H - 1);
+        s_gy[t][0] = pre::axis_sample(first, p.src_h, p.H).i0;
+        s_gy[t][1] = pre::axis_sample(last, p.src_h, p.H).i1;
+      }
+    }
+  }
   fence_proxy_async_smem();
   if (warp == 4) {
     __syncwarp();   // the weight-staging loop may have left the lanes apart; the allocation is warp-collective
@@ -90,6 +151,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
 
   const int tiles_per_img = p.tiles_x * p.tiles_y;
   const int total_tiles = p.K * tiles_per_img;
+  const float inv_tiles_x = 1.0f / (float)p.tiles_x, inv_tiles_per_img = 1.0f / (float)tiles_per_img;
 
   if (warp < 4) {
     // ------------------------------------------------------------------ operand producers
@@ -110,7 +172,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
     };
 
     bool fail = false;   // a bounded wait ran out; the four warps learn of it together at the barrier
-    if (ptid == 0) {
+    if (!FUSED && ptid == 0) {
       if (blockIdx.x < total_tiles) fetch_patch(blockIdx.x, 0);
       if (blockIdx.x + gridDim.x < total_tiles) fetch_patch(blockIdx.x + gridDim.x, 1);
     }
@@ -126,8 +188,9 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
           for (int kx = 0; kx < 3; ++kx)
             v[(c * 3 + ky) * 3 + kx] = patch[(c * PH + py * STRIDE + ky) * BW + px * STRIDE + kx + 3];
       // the four producer warps meet here: everybody has read this patch buffer, it can be refilled
+      if (FUSED) mbar_arrive(smem_u32(p_empty + buf));
       if (named_barrier_or(1, 128, fail)) break;
-      if (ptid == 0 && tile + 2 * (int)gridDim.x < total_tiles) {
+      if (!FUSED && ptid == 0 && tile + 2 * (int)gridDim.x < total_tiles) {
         fence_proxy_async_smem();
         fetch_patch(tile + 2 * gridDim.x, buf);
       }
@@ -176,6 +239,117 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
+  } else if (FUSED && warp >= 9) {
+    // ------------------------------------------------------- frame samplers (preprocessing)
+    // Patch entry (c, r, j + 3) is pixel (y_base + r, x_base + j) of the resized image, zero outside it (the
+    // convolution's padding).  Thread (g, j) of the first RG * PW owns patch column j and the rows g, g + RG, ...:
+    // its horizontal sample position is worked out once per tile and stays in registers.  The next PH threads work
+    // out the vertical positions of the tile's rows into shared memory meanwhile (one integer division per thread).
+    //
+    // Staging: in pass k thread t moves 16-byte vector t % 16 of footprint row t / 16 + 8k.  The stage written
+    // while tile i is handled (for tile i + 2) was last read for tile i - 1, which every thread has left behind
+    // at tile i's barrier; the same barrier, one tile later, makes the stores visible before they are read.
+    constexpr int RG = (128 - PH) / PW;
+    constexpr int ROWS = (PH + RG - 1) / RG;
+    const int bt = threadIdx.x - F_THREADS;
+    const int g = bt / PW, j = bt - g * PW;
+    const int stage_bytes = p.src_rows_cap * p.src_row_cap;
+    const int vrow = bt >> 4, vcol = bt & 15;
+    const float inv_den_x = 1.0f / (float)(2 * p.W), inv_den_y = 1.0f / (float)(2 * p.H);
+    uint4 vreg[F_SRC_PASSES];
+    uint32_t vmask = 0;
+    uint32_t st = 0;   // stage of the current tile's rows
+
+    auto stage_load = [&](int tile) {
+      const TileAt t = tile_at(tile, p.tiles_x, tiles_per_img, inv_tiles_x, inv_tiles_per_img);
+      const int sx_lo = s_gx[t.tx][0], sx_hi = s_gx[t.tx][1], sy_lo = s_gy[t.ty][0], sy_hi = s_gy[t.ty][1];
+      const int n_rows = min(sy_hi - sy_lo + 1, p.src_rows_cap);
+      const int span = 3 * (sx_hi - sx_lo) + 2;            // a row's bytes run from its first byte to first + span
+      uintptr_t g_first = (uintptr_t)s_frame[t.img] + (size_t)(sy_lo + vrow) * p.src_pitch + (size_t)3 * sx_lo;
+      vmask = 0;
+#pragma unroll
+      for (int k = 0; k < F_SRC_PASSES; ++k) {
+        const uintptr_t a_vec = (g_first & ~(uintptr_t)15) + (uintptr_t)vcol * 16;
+        // the vector starts at or before the row's last byte and inside the staged row
+        if (vrow + 8 * k < n_rows && a_vec <= g_first + span && vcol < (p.src_row_cap >> 4)) {
+          vreg[k] = __ldg(reinterpret_cast<const uint4*>(a_vec));
+          vmask |= 1u << k;
+        }
+        g_first += (size_t)8 * p.src_pitch;
+      }
+    };
+    auto stage_store = [&](int st) {
+      uint8_t* dst = s_src + st * stage_bytes + vrow * p.src_row_cap + vcol * 16;
+#pragma unroll
+      for (int k = 0; k < F_SRC_PASSES; ++k)
+        if (vmask & (1u << k)) *reinterpret_cast<uint4*>(dst + 8 * k * p.src_row_cap) = vreg[k];
+    };
+
+    // the first two tiles' rows
+    if (blockIdx.x < total_tiles) { stage_load(blockIdx.x); stage_store(0); }
+    if (blockIdx.x + gridDim.x < total_tiles) { stage_load(blockIdx.x + gridDim.x); stage_store(1); }
+    uint32_t it = 0;
+    bool fail = false;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+      const int b = (int)(it & 1u);
+      const TileAt t = tile_at(tile, p.tiles_x, tiles_per_img, inv_tiles_x, inv_tiles_per_img);
+      const int x_base = t.tx * 16 * STRIDE - 1, y_base = t.ty * 8 * STRIDE - 1;
+      const int sx_lo = s_gx[t.tx][0], sy_lo = s_gy[t.ty][0];
+      const bool ahead = tile + 2 * (int)gridDim.x < total_tiles;
+      if (ahead) stage_load(tile + 2 * gridDim.x);
+      int xo = -1;
+      float fx = 0.f;
+      if (g < RG) {
+        const int x = x_base + j;
+        if (x >= 0 && x < p.W) {
+          const pre::AxisSample sx = pre::axis_sample_fast(x, p.src_w, p.W, inv_den_x);
+          xo = 3 * (sx.i0 - sx_lo);
+          fx = sx.f;
+        }
+      } else if (bt < RG * PW + PH) {
+        const int r = bt - RG * PW, y = y_base + r;
+        const bool in = y >= 0 && y < p.H;
+        const pre::AxisSample sy = pre::axis_sample_fast(in ? y : 0, p.src_h, p.H, inv_den_y);
+        const uint32_t src_lo = (uint32_t)(uintptr_t)s_frame[t.img];   // only the low bits matter for 16-byte alignment
+        // byte position of source column sx_lo inside the two staged rows
+        s_yoff0[b][r] = in ? (sy.i0 - sy_lo) * p.src_row_cap + (int)((src_lo + (uint32_t)(sy.i0 * p.src_pitch + 3 * sx_lo)) & 15u) : -1;
+        s_yoff1[b][r] = in ? (sy.i1 - sy_lo) * p.src_row_cap + (int)((src_lo + (uint32_t)(sy.i1 * p.src_pitch + 3 * sx_lo)) & 15u) : -1;
+        s_fy[b][r] = sy.f;
+      }
+      if (!mbar_wait(smem_u32(p_empty + b), ((it >> 1) & 1u) ^ 1u, abort_flag, p.status, 0xA00 + b, wait_limit)) fail = true;
+      if (named_barrier_or(4, 128, fail)) break;
+      if (g < RG) {
+        const uint32_t* words = reinterpret_cast<const uint32_t*>(s_src + st * stage_bytes);
+        float* d = reinterpret_cast<float*>(s_patch + b * PATCH_STRIDE) + j + 3;
+#pragma unroll
+        for (int k = 0; k < ROWS; ++k) {
+          // rows behind the patch's last are computed like the last one and not stored; samples outside the image
+          // are computed from the first staged bytes and replaced by zero: no branch but the one on fy
+          const int r = g + k * RG, rc = min(r, PH - 1);
+          const int y0 = s_yoff0[b][rc];
+          const float fy = s_fy[b][rc];
+          const bool in = xo >= 0 && y0 >= 0;
+          float o0, o1, o2;
+          uint32_t lo0, hi0;
+          fetch_pair(words, in ? y0 + xo : 0, lo0, hi0);
+          if (fy == 0.0f) {
+            pre::sample_row(lo0, hi0, fx, p.scale, p.shift, o0, o1, o2);
+          } else {
+            uint32_t lo1, hi1;
+            fetch_pair(words, in ? s_yoff1[b][rc] + xo : 0, lo1, hi1);
+            pre::sample_rows(lo0, hi0, lo1, hi1, fx, fy, p.scale, p.shift, o0, o1, o2);
+          }
+          if (r < PH) {
+            d[r * BW] = in ? o0 : 0.f;
+            d[(PH + r) * BW] = in ? o1 : 0.f;
+            d[(2 * PH + r) * BW] = in ? o2 : 0.f;
+          }
+        }
+      }
+      mbar_arrive(smem_u32(p_full + b));
+      if (ahead) stage_store((int)(st == 0 ? 2 : st - 1));   // (it + 2) mod 3
+      st = st == 2 ? 0 : st + 1;
+    }
   } else {
     // --------------------------------------------------------------------------- epilogue
     const int quarter = warp & 3;
@@ -187,7 +361,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
     uint32_t acc_phase = 0;
     int acc = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, img = tile / tiles_per_img;
+      const TileAt t = tile_at(tile, p.tiles_x, tiles_per_img, inv_tiles_x, inv_tiles_per_img);
       const bool fail = !mbar_wait(smem_u32(t_full + acc), acc_phase, abort_flag, p.status, 0x800 + acc, wait_limit);
       // the previous tile's store must have finished reading s_out before it is overwritten
       if (leader) bulk_wait_group_read0();
@@ -219,7 +393,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
       fence_proxy_async_smem();
       asm volatile("bar.sync 3, 128;" ::: "memory");
       if (leader) {
-        tma_store_4d(&p.map_out, smem_u32(s_out), 0, tx * 16, ty * 8, img);
+        tma_store_4d(&p.map_out, smem_u32(s_out), 0, t.tx * 16, t.ty * 8, t.img);
         bulk_commit_group();
       }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
@@ -240,20 +414,51 @@ __global__ void __launch_bounds__(F_THREADS, 3) conv_first_tc_kernel(const __gri
   }
 }
 
-template <int COUT, int STRIDE>
-cudaError_t launch_t(const ConvFirstTcParams& p, int grid, cudaStream_t s) {
+template <int COUT, int STRIDE, bool FUSED>
+cudaError_t launch_t(const ConvFirstTcParams& p, int sm_count, cudaStream_t s) {
   constexpr int PH = 7 * STRIDE + 3;
   constexpr int SMEM = 1024 + 128 * COUT * 2 + F_STAGES * F_A_BYTES + COUT * 64 + 2 * ((3 * PH * box_w(STRIDE) * 4 + 127) & ~127);
-  auto kern = conv_first_tc_kernel<COUT, STRIDE>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  const int smem = SMEM + (FUSED ? F_SRC_STAGES * p.src_rows_cap * p.src_row_cap : 0);
+  const int total = p.K * p.tiles_x * p.tiles_y;
+  const int slots = (FUSED ? 2 : 3) * sm_count;
+  const int grid = total < slots ? total : slots;
+  auto kern = conv_first_tc_kernel<COUT, STRIDE, FUSED>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FUSED ? SMEM + F_SRC_BUDGET : SMEM);
   if (e != cudaSuccess) return e;
-  return launch_kernel(kern, grid, F_THREADS, SMEM, s, p, p.pdl != 0);
+  return launch_kernel(kern, grid, FUSED ? F_THREADS_FUSED : F_THREADS, smem, s, p, p.pdl != 0);
+}
+
+template <bool FUSED>
+cudaError_t launch_f(const ConvFirstTcParams& p, int sm_count, cudaStream_t s) {
+  if (p.cout == 32 && p.stride == 1) return launch_t<32, 1, FUSED>(p, sm_count, s);
+  if (p.cout == 32 && p.stride == 2) return launch_t<32, 2, FUSED>(p, sm_count, s);
+  if (p.cout == 64 && p.stride == 1) return launch_t<64, 1, FUSED>(p, sm_count, s);
+  if (p.cout == 64 && p.stride == 2) return launch_t<64, 2, FUSED>(p, sm_count, s);
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace
 
 bool conv_first_tc_supported(int cout) { return cout == 32 || cout == 64; }
 int conv_first_tc_box_w(int stride) { return box_w(stride); }
+
+bool conv_first_tc_staging(int stride, int src_w, int src_h, int net_w, int net_h, int* rows_cap, int* row_cap) {
+  const int wo = (net_w + stride - 1) / stride, ho = (net_h + stride - 1) / stride;
+  if ((wo + 15) / 16 > F_MAX_TILES || (ho + 7) / 8 > F_MAX_TILES) return false;
+  // Worst-case footprint of a (7*stride+3) x (15*stride+3) patch: rows = ceil(PH * sh/nh) + 2; bytes per row =
+  // 3 * (ceil(PW * sw/nw) + 2) + 15 (alignment at the front) + 15 (at the end) + 12 (the tap fetch reads three
+  // whole words from its first byte), rounded up to 16.
+  const long ph = 7 * stride + 3, pw = 15 * stride + 3;
+  const long rows = (ph * src_h + net_h - 1) / net_h + 2;
+  const long cols = (pw * src_w + net_w - 1) / net_w + 2;
+  const long cap = ((3 * cols + 48 + 15) / 16) * 16;
+  *rows_cap = (int)rows;
+  *row_cap = (int)cap;
+  if (rows > 8 * F_SRC_PASSES || cap > 256) return false;   // what the staging passes of the kernel cover
+  // the sample positions are worked out with pre::div_by: numerators below 2^27
+  if ((2L * net_w + 1) * src_w >= (1L << 27) || (2L * net_h + 1) * src_h >= (1L << 27)) return false;
+  return F_SRC_STAGES * rows * cap <= F_SRC_BUDGET;
+}
 
 // [cout][27] bf16 bit patterns (row-major, k = c*9 + ky*3 + kx) -> operand layout, cout*32 values
 void conv_first_tc_pack(const uint16_t* w_bf16, int cout, uint16_t* packed) {
@@ -263,13 +468,7 @@ void conv_first_tc_pack(const uint16_t* w_bf16, int cout, uint16_t* packed) {
 }
 
 cudaError_t launch_conv_first_tc(const ConvFirstTcParams& p, int sm_count, cudaStream_t s) {
-  const int total = p.K * p.tiles_x * p.tiles_y;
-  const int grid = total < 3 * sm_count ? total : 3 * sm_count;
-  if (p.cout == 32 && p.stride == 1) return launch_t<32, 1>(p, grid, s);
-  if (p.cout == 32 && p.stride == 2) return launch_t<32, 2>(p, grid, s);
-  if (p.cout == 64 && p.stride == 1) return launch_t<64, 1>(p, grid, s);
-  if (p.cout == 64 && p.stride == 2) return launch_t<64, 2>(p, grid, s);
-  return cudaErrorInvalidValue;
+  return p.fused ? launch_f<true>(p, sm_count, s) : launch_f<false>(p, sm_count, s);
 }
 
 }  // namespace tt

@@ -9,34 +9,18 @@
 // fetched as three 32-bit shared loads plus funnel shifts, bytes become floats by a byte
 // permute into the mantissa of 2^23, and the results leave as three 128-bit stores.
 #include "tt_internal.h"
+#include "pre_math.cuh"
 
 namespace tt {
 namespace {
+
+using namespace pre;
 
 constexpr int PRE_TX = 32;          // threads along x; each makes 4 outputs -> 128 outputs per block row
 constexpr int PRE_TY = 8;           // output rows per block
 constexpr int PRE_OUT_W = PRE_TX * 4;
 constexpr int PRE_THREADS = PRE_TX * PRE_TY;
 constexpr int PRE_SMEM_BYTES = 44 * 1024;
-
-struct AxisSample {
-  int i0, i1;
-  float f;
-};
-
-// Exact integer evaluation of s = clamp((o + 1/2) * in/out - 1/2, 0, in - 1):
-// s = num/den with num = (2o+1)*in - out, den = 2*out.
-__device__ __forceinline__ AxisSample axis_sample(int o, int in, int out) {
-  int den = 2 * out;
-  int num = (2 * o + 1) * in - out;
-  int hi = (in - 1) * den;
-  num = max(0, min(num, hi));
-  AxisSample r;
-  r.i0 = num / den;
-  r.i1 = min(r.i0 + 1, in - 1);
-  r.f = (float)(num - r.i0 * den) / (float)den;  // both integers are exact in fp32
-  return r;
-}
 
 // Six bytes starting at byte offset `b` of a word-aligned shared buffer: the RGB triples of two
 // neighbouring pixels.  lo = bytes b..b+3 (R0 G0 B0 R1), hi = bytes b+4..b+7 (G1 B1 . .).
@@ -46,21 +30,6 @@ __device__ __forceinline__ void fetch_pair(const uint32_t* s_words, int b, uint3
   const uint32_t w0 = s_words[w], w1 = s_words[w + 1], w2 = s_words[w + 2];
   lo = __funnelshift_r(w0, w1, sh);
   hi = __funnelshift_r(w1, w2, sh);
-}
-
-// byte k of x as the float 2^23 + b (exact)
-__device__ __forceinline__ float byte_to_magic(uint32_t x, uint32_t selector) {
-  return __uint_as_float(__byte_perm(x, 0x4B000000u, selector));
-}
-
-// Bilinear blend of four taps given as 2^23 + byte, then the normalisation as one fused
-// multiply-add.  Differences of two such floats are the exact byte differences, so only the
-// left taps need the 2^23 removed.
-__device__ __forceinline__ float blend_magic(float l0, float r0, float l1, float r1, float fx, float fy, float scale,
-                                             float shift) {
-  const float top = fmaf(fx, r0 - l0, l0 - 8388608.0f);
-  const float bot = fmaf(fx, r1 - l1, l1 - 8388608.0f);
-  return fmaf(fmaf(fy, bot - top, top), scale, shift);
 }
 
 constexpr int PRE_ROWS = 16;          // output rows per block of the staged kernel: 2 per thread
@@ -73,6 +42,9 @@ preprocess_staged_kernel(const __grid_constant__ PreprocessParams p, int row_cap
   __shared__ int s_y0[PRE_ROWS], s_y1[PRE_ROWS];     // source rows of every output row of the tile
   __shared__ float s_fy[PRE_ROWS];
   __shared__ int s_xlo, s_xhi;                       // source column range of the tile
+  // the next kernel of the stream, if it was launched as a programmatic dependent, may start its set-up now;
+  // it waits for this grid to finish before it reads the output
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int n = blockIdx.z;
   const uint8_t* __restrict__ src = p.src_tab ? p.src_tab[n] : p.src.p[n];
   const uint32_t src_lo = (uint32_t)(uintptr_t)src;  // only the low bits matter for 16-byte alignment
@@ -143,9 +115,7 @@ preprocess_staged_kernel(const __grid_constant__ PreprocessParams p, int row_cap
       for (int j = 0; j < 4; ++j) {
         uint32_t lo0, hi0;
         fetch_pair(s_words, base0 + xoffs[j], lo0, hi0);
-        o0[j] = fmaf(fmaf(fxs[j], byte_to_magic(lo0, 0x7443) - byte_to_magic(lo0, 0x7440), byte_to_magic(lo0, 0x7440) - 8388608.0f), scale, shift);
-        o1[j] = fmaf(fmaf(fxs[j], byte_to_magic(hi0, 0x7440) - byte_to_magic(lo0, 0x7441), byte_to_magic(lo0, 0x7441) - 8388608.0f), scale, shift);
-        o2[j] = fmaf(fmaf(fxs[j], byte_to_magic(hi0, 0x7441) - byte_to_magic(lo0, 0x7442), byte_to_magic(lo0, 0x7442) - 8388608.0f), scale, shift);
+        sample_row(lo0, hi0, fxs[j], scale, shift, o0[j], o1[j], o2[j]);
       }
     } else {
 #pragma unroll
@@ -153,13 +123,7 @@ preprocess_staged_kernel(const __grid_constant__ PreprocessParams p, int row_cap
         uint32_t lo0, hi0, lo1, hi1;
         fetch_pair(s_words, base0 + xoffs[j], lo0, hi0);
         fetch_pair(s_words, base1 + xoffs[j], lo1, hi1);
-        // channel c of the left pixel is byte c of lo; of the right pixel: byte 3 of lo, bytes 0, 1 of hi
-        o0[j] = blend_magic(byte_to_magic(lo0, 0x7440), byte_to_magic(lo0, 0x7443), byte_to_magic(lo1, 0x7440),
-                            byte_to_magic(lo1, 0x7443), fxs[j], fy, scale, shift);
-        o1[j] = blend_magic(byte_to_magic(lo0, 0x7441), byte_to_magic(hi0, 0x7440), byte_to_magic(lo1, 0x7441),
-                            byte_to_magic(hi1, 0x7440), fxs[j], fy, scale, shift);
-        o2[j] = blend_magic(byte_to_magic(lo0, 0x7442), byte_to_magic(hi0, 0x7441), byte_to_magic(lo1, 0x7442),
-                            byte_to_magic(hi1, 0x7441), fxs[j], fy, scale, shift);
+        sample_rows(lo0, hi0, lo1, hi1, fxs[j], fy, scale, shift, o0[j], o1[j], o2[j]);
       }
     }
     float* d0 = p.dst + (size_t)n * 3 * plane + (size_t)yo * p.net_w + xo0;
@@ -211,8 +175,7 @@ __global__ void __launch_bounds__(PRE_THREADS) preprocess_direct_kernel(const __
 
 cudaError_t launch_preprocess(const PreprocessParams& p, cudaStream_t s) {
   dim3 block(PRE_TX, PRE_TY);
-  // ((v / div) - mean) / std as one fused multiply-add: v * scale + shift
-  const float scale = p.inv_div * p.inv_std, shift = -p.mean * p.inv_std;
+  const float scale = pre::norm_scale(p.inv_div, p.inv_std), shift = pre::norm_shift(p.mean, p.inv_std);
   // Worst-case staged footprint of one block: rows = ceil(TY * sh/nh) + 2; bytes per row =
   // 3 * (ceil(OUT_W * sw/nw) + 2) + 15 (alignment at the front) + 15 (at the end) + 12 (the tap
   // fetch reads three whole words from its first byte), rounded up to 16.

@@ -16,6 +16,7 @@
 #include <vector>
 
 #include "tt_internal.h"
+#include "pre_math.cuh"
 
 using namespace tt;
 
@@ -114,6 +115,8 @@ struct tt_ctx {
   bool use_post_tc = false;
   ConvFirstTcParams first_tc{}; // bf16 path, first encoder layer on the tensor cores when its width (32 or 64) allows
   bool use_first_tc = false;
+  bool fuse_pre = false;        // the first layer samples the frames itself; no preprocess launch, ctx->pre is not written
+  FramePtrs fp_inflight{};      // device frame pointers of the submit being described (saved per slot)
   SimtLayer simt_enc[TT_MAX_ENC];
   SimtLayer simt_lstm;
   TcLayer tc_enc[TT_MAX_ENC];
@@ -132,6 +135,7 @@ struct tt_ctx {
     cudaEvent_t ev_start = nullptr, ev_stop = nullptr, ev_copy = nullptr;
     cudaEvent_t stage_ev[TT_STAGE_COUNT + 1] = {};
     bool stage_ran[TT_STAGE_COUNT] = {};
+    FramePtrs fp{};
     bool profiled = false;
     int K = 0;
     tt_frame frames[TT_MAX_STREAMS];
@@ -210,6 +214,7 @@ void bind_slot(tt_ctx* ctx, int i) {
   ctx->tick_profiled = sl.profiled;
   ctx->K_inflight = sl.K;
   for (int k = 0; k < TT_MAX_STREAMS; ++k) { ctx->frames_inflight[k] = sl.frames[k]; ctx->states_inflight[k] = sl.states[k]; }
+  ctx->fp_inflight = sl.fp;
   ctx->bound = i;
 }
 
@@ -223,6 +228,7 @@ void save_slot(tt_ctx* ctx, int i) {
   sl.profiled = ctx->tick_profiled;
   sl.K = ctx->K_inflight;
   for (int k = 0; k < TT_MAX_STREAMS; ++k) { sl.frames[k] = ctx->frames_inflight[k]; sl.states[k] = ctx->states_inflight[k]; }
+  sl.fp = ctx->fp_inflight;
 }
 
 #define TT_CUDA(ctx, expr)                                                                         \
@@ -582,6 +588,12 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
         if ((st = encode_map_f32(ctx, &f.map_in, ctx->pre, 4, dims, str, box)) != TT_OK) return st;
       }
       ctx->use_first_tc = true;
+      ctx->fuse_pre = c.options[TT_OPT_FUSED_PRE] != 0 &&
+                      conv_first_tc_staging(f.stride, c.src_w, c.src_h, c.net_w, c.net_h, &f.src_rows_cap, &f.src_row_cap);
+      f.fused = ctx->fuse_pre ? 1 : 0;
+      f.src_w = c.src_w; f.src_h = c.src_h; f.src_pitch = c.src_pitch;
+      f.scale = pre::norm_scale(1.0f / c.norm_div, 1.0f / c.norm_std);
+      f.shift = pre::norm_shift(c.norm_mean, 1.0f / c.norm_std);
     } else if ((st = pack_simt(ctx, &ctx->simt_enc[0], w->enc_w[0], w->enc_b[0], 3, ctx->lay_c[1], c.enc_stride[0],
                                ctx->lay_c[1] > 16 ? 32 : 16, 0, true)) != TT_OK) {
       return st;
@@ -694,6 +706,16 @@ tt_status mark_stage(tt_ctx* ctx, int stage, int launches) {
   return TT_OK;
 }
 
+PreprocessParams preprocess_params(const tt_ctx* ctx, int K, const FramePtrs& frames, const uint8_t* const* tab) {
+  const tt_config& c = ctx->cfg;
+  PreprocessParams pp;
+  pp.src = frames; pp.src_tab = tab; pp.K = K; pp.src_w = c.src_w; pp.src_h = c.src_h; pp.src_pitch = c.src_pitch;
+  pp.net_w = c.net_w; pp.net_h = c.net_h;
+  pp.inv_div = 1.0f / c.norm_div; pp.mean = c.norm_mean; pp.inv_std = 1.0f / c.norm_std;
+  pp.dst = ctx->pre;
+  return pp;
+}
+
 // Launch sequence of one tick.  Everything is enqueued on ctx->stream.
 tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* const* states) {
   const tt_config& c = ctx->cfg;
@@ -709,13 +731,10 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
     h_out.v[n] = slot * 2 + (1 - half);
   }
 
-  PreprocessParams pp;
-  pp.src = frames; pp.src_tab = ctx->cur_tab; pp.K = K; pp.src_w = c.src_w; pp.src_h = c.src_h; pp.src_pitch = c.src_pitch;
-  pp.net_w = c.net_w; pp.net_h = c.net_h;
-  pp.inv_div = 1.0f / c.norm_div; pp.mean = c.norm_mean; pp.inv_std = 1.0f / c.norm_std;
-  pp.dst = ctx->pre;
-  TT_CUDA(ctx, launch_preprocess(pp, s));
-  if ((ms_ = mark_stage(ctx, TT_STAGE_PREPROCESS, 1)) != TT_OK) return ms_;
+  if (!ctx->fuse_pre) {
+    TT_CUDA(ctx, launch_preprocess(preprocess_params(ctx, K, frames, ctx->cur_tab), s));
+    if ((ms_ = mark_stage(ctx, TT_STAGE_PREPROCESS, 1)) != TT_OK) return ms_;
+  }
 
   if (!ctx->bf16) {
     const float* in = ctx->pre;
@@ -747,7 +766,9 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
   } else {
     if (ctx->use_first_tc) {
       ctx->first_tc.K = K;
-      ctx->first_tc.pdl = ctx->profiling ? 0 : 1;
+      // with the preprocessing inside it the kernel is the first of the tick and may follow a copy: launched normally
+      ctx->first_tc.pdl = (ctx->profiling || ctx->fuse_pre) ? 0 : 1;
+      ctx->first_tc.src = frames; ctx->first_tc.src_tab = ctx->cur_tab;
       TT_CUDA(ctx, launch_conv_first_tc(ctx->first_tc, ctx->sm_count, s));
       if ((ms_ = mark_stage(ctx, TT_STAGE_ENC0, 1)) != TT_OK) return ms_;
     } else {
@@ -1125,6 +1146,7 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
     states[n]->last_pos = n;
   }
   ctx->K_inflight = K;
+  ctx->fp_inflight = fp;
   save_slot(ctx, slot);
   ctx->q_count += 1;
   return TT_OK;
@@ -1217,6 +1239,10 @@ tt_status tt_debug_tensor(tt_ctx* ctx, tt_state* st, int32_t which, float* host_
   bind_slot(ctx, ctx->last_done);
   if (which == TT_TENSOR_PRE) {
     n = (size_t)3 * ctx->cfg.net_h * ctx->cfg.net_w;
+    if (ctx->fuse_pre) {
+      // the resized image never reached memory: make it now, from the frame buffers of that submit
+      TT_CUDA(ctx, launch_preprocess(preprocess_params(ctx, ctx->K_inflight, ctx->fp_inflight, nullptr), s));
+    }
     src = ctx->pre + (size_t)pos * n;
   } else if (which >= TT_TENSOR_ENC0 && which < TT_TENSOR_ENC0 + ctx->n_enc) {
     const int l = which - TT_TENSOR_ENC0;

@@ -99,8 +99,19 @@ struct ConvFirstTcParams {
   const float* bias;          // device, [cout]
   int32_t* status;
   long long wait_limit;       // SM cycles after which a barrier wait gives up
+  // fused preprocessing: the kernel samples the uint8 RGB frames itself (resize to W x H, then v * scale + shift)
+  // and neither `in` nor map_in is used
+  int32_t fused;
+  FramePtrs src;                   // frame pointers by value ...
+  const uint8_t* const* src_tab;   // ... or, if non-null, a device table of them
+  int32_t src_w, src_h, src_pitch;
+  float scale, shift;
+  int32_t src_rows_cap, src_row_cap;   // staged frame rows per tile and bytes per staged row (conv_first_tc_staging)
 };
 bool conv_first_tc_supported(int cout);
+// Shared-memory footprint of the frame rows one tile of the fused form stages: rows and bytes per row
+// (a multiple of 16).  False if the resize factor makes it too large; the preprocessing then stays a kernel of its own.
+bool conv_first_tc_staging(int stride, int src_w, int src_h, int net_w, int net_h, int* rows_cap, int* row_cap);
 int conv_first_tc_box_w(int stride);   // columns of the input patch box (a multiple of 4)
 void conv_first_tc_pack(const uint16_t* w_bf16, int cout, uint16_t* packed);
 cudaError_t launch_conv_first_tc(const ConvFirstTcParams& p, int sm_count, cudaStream_t s);

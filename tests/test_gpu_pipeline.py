@@ -13,10 +13,11 @@ from parity_util import assert_close, check_masks, check_reductions_from_own_mas
 pytestmark = pytest.mark.gpu
 
 
-def _make(wl, K=1, overlay=None, precision=None, timeout_ns=0, plain_launches=False, cta_pairs=False, halo=True):
+def _make(wl, K=1, overlay=None, precision=None, timeout_ns=0, plain_launches=False, cta_pairs=False, halo=True,
+          fused_pre=False):
     weights = tt_synth.make_weights(wl)
     cfg = binding.make_config(wl, max_streams=K, overlay=overlay, precision=precision, sync_timeout_ns=timeout_ns,
-                              plain_launches=plain_launches, cta_pairs=cta_pairs, halo=halo)
+                              plain_launches=plain_launches, cta_pairs=cta_pairs, halo=halo, fused_pre=fused_pre)
     ctx = binding.Context(cfg, weights)
     states = [ctx.state_create() for _ in range(K)]
     return ctx, states, weights
@@ -302,6 +303,50 @@ def test_bf16_convlstm_one_box_per_tap_still_matches(cuda_device):
         ctx.destroy()
     for a, b in zip(*outs):
         assert rms_err(a, b) < 1e-3
+
+
+@pytest.mark.parametrize("shape", [
+    dict(src_w=214, src_h=120, net_w=160, net_h=120),                 # one axis resized, ragged tiles
+    dict(src_w=203, src_h=157, net_w=132, net_h=100),                 # both axes resized, odd pitch, partial tiles
+    dict(src_w=96, src_h=64, net_w=128, net_h=96),                    # up-scaling
+    dict(src_w=160, src_h=120, net_w=160, net_h=120, stride1=True),   # no resize, stride-1 first layer
+])
+def test_bf16_preprocessing_inside_the_first_layer_changes_no_bit(cuda_device, shape):
+    """On request the first encoder layer samples the frames itself; against the preprocessing as a kernel of its own
+    (which writes the resized fp32 image the layer then reads) every output and the state must be the same bits.
+    Stream 1's frames sit at an odd address, and the last frame ends where its buffer ends."""
+    shape = dict(shape)
+    stride1 = shape.pop("stride1", False)
+    wl = tt_synth.workload("cfg1-gain").with_(name="fuse", overlay=True, **shape)
+    if stride1:
+        wl = wl.with_(enc_stride=(1,) + tuple(wl.enc_stride[1:]))
+    K, n = 2, 3
+    host = _frames(wl, K, n)
+    nbytes = host[0][0].size
+    runs = []
+    for fused in (True, False):
+        ctx, states, _ = _make(wl, K, overlay=True, fused_pre=fused)
+        out = []
+        for t in range(n):
+            bufs = [torch.empty(nbytes + 1, dtype=torch.uint8, device=cuda_device) for _ in range(K)]
+            views = []
+            for k in range(K):
+                v = bufs[k][k:k + nbytes]          # stream 1: odd address, last byte of the frame = last byte of the buffer
+                v.copy_(torch.from_numpy(host[k][t]).reshape(-1))
+                views.append(v.view(host[k][t].shape))
+            ctx.submit_frames(views, states, frame_index=t)
+            res = ctx.sync()
+            out.append([(ctx.fetch_probs(r), ctx.fetch_masks(r), ctx.fetch_overlay(r), r["conf"].copy(), r["cx"].copy(),
+                         ctx.debug_tensor(states[i], "pre"), ctx.debug_tensor(states[i], "enc0")) for i, r in enumerate(res)])
+        runs.append((out, [ctx.state_export(s) for s in states]))
+        ctx.destroy()
+    (a, ha), (b, hb) = runs
+    for ta, tb in zip(a, b):
+        for ra, rb in zip(ta, tb):
+            for va, vb in zip(ra, rb):
+                assert np.array_equal(va, vb)
+    for (h1, c1), (h2, c2) in zip(ha, hb):
+        assert np.array_equal(h1, h2) and np.array_equal(c1, c2)
 
 
 def test_bf16_eight_tools_and_mean_sigmoid_confidence(cuda_device):
