@@ -35,6 +35,7 @@ extern "C" {
 #define TT_MAX_STREAMS 8
 #define TT_MAX_TOOLS 8
 #define TT_MAX_ENC 4
+#define TT_MAX_IN_FLIGHT 3   /* submits that may be in flight in one context */
 
 typedef enum {
   TT_OK = 0,
@@ -43,7 +44,7 @@ typedef enum {
   TT_ERR_OOM = 3,           /* device or host allocation failed */
   TT_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed; see tt_last_error */
   TT_ERR_ADMISSION = 5,     /* more streams than the context was sized for (Section IV-A, admission control) */
-  TT_ERR_NOT_READY = 6,     /* submit while two submits are in flight, sync with nothing submitted, state access while in flight */
+  TT_ERR_NOT_READY = 6,     /* submit while TT_MAX_IN_FLIGHT submits are in flight, sync with nothing submitted, state access while in flight */
   TT_ERR_TIMEOUT = 7,       /* bounded wait expired; the device is left usable */
   TT_ERR_DEVICE_STATUS = 8  /* a kernel reported a bounded device-side wait that ran out */
 } tt_status;
@@ -141,7 +142,7 @@ typedef struct {
   float cx[TT_MAX_TOOLS];      /* mask centroid in mask-grid index coordinates; -1 when the mask is empty */
   float cy[TT_MAX_TOOLS];
   int32_t count[TT_MAX_TOOLS]; /* pixels above threshold */
-  const uint8_t* masks_dev;    /* device, [n_tools][Hm][Wm] 0/1; valid until the second submit after this one */
+  const uint8_t* masks_dev;    /* device, [n_tools][Hm][Wm] 0/1; valid until submit number TT_MAX_IN_FLIGHT after this one */
   const float* probs_dev;      /* device, [n_tools][Hm][Wm]; same lifetime */
   const uint8_t* overlay_dev;  /* device, [src_h][src_w][4] RGBA8, or NULL when overlay is off */
   float gpu_ms;                /* device time of the whole batch this frame was part of */
@@ -193,11 +194,12 @@ tt_status tt_state_import(tt_ctx* ctx, tt_state* st, const float* h_host, const 
  *   S5 per tool     confidence (mean of p, or sigmoid(linear(global-average-pool(h')))),
  *                   count and centroid of the mask;
  *   S6 overlay      (if enabled) alpha-0.4 integer blend of the masks onto an RGBA8 copy.
- * Asynchronous: returns once the work is enqueued.  Up to two submits may be in flight (the
- * host->device copy of the second overlaps the compute of the first; ticks execute in submit
- * order, so a state may be used by both); tt_sync returns them oldest first.  frames[k].data must
+ * Asynchronous: returns once the work is enqueued.  Up to TT_MAX_IN_FLIGHT submits may be in flight (the
+ * host->device copies of the later ones overlap the compute of the first: with three, the copy engine
+ * need not wait for the host between ticks; ticks execute in submit order, so a state may be used by
+ * all of them); tt_sync returns them oldest first.  frames[k].data must
  * stay valid until the tt_sync of its submit returns.  Errors: K < 1 or null/duplicate/foreign states -> TT_ERR_INVALID_ARG;
- * K > max_streams -> TT_ERR_ADMISSION; two submits already in flight -> TT_ERR_NOT_READY.
+ * K > max_streams -> TT_ERR_ADMISSION; TT_MAX_IN_FLIGHT submits already in flight -> TT_ERR_NOT_READY.
  * Nothing is enqueued when one of these argument errors is returned.
  */
 tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_state* const* states);

@@ -14,6 +14,7 @@ import numpy as np
 
 TT_ABI_VERSION = 1
 TT_MAX_STREAMS = 8
+TT_MAX_IN_FLIGHT = 3
 TT_MAX_TOOLS = 8
 TT_MAX_ENC = 4
 

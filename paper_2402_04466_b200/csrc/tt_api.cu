@@ -123,9 +123,9 @@ struct tt_ctx {
   TcLayer tc_lstm;
 
   tt_state states[TT_MAX_STREAMS];
-  // Up to two submits may be in flight.  Everything a tick owns (frame staging, outputs, result
-  // blocks, events) exists twice; the members above/below named like the slot's are the slot that
-  // is currently bound (bind_slot / save_slot).
+  // Up to TT_MAX_IN_FLIGHT submits may be in flight.  Everything a tick owns (frame staging, outputs,
+  // result blocks, events) exists once per slot; the members above/below named like the slot's are the
+  // slot that is currently bound (bind_slot / save_slot).
   struct Slot {
     uint8_t* frames_stage = nullptr;
     float *logits = nullptr, *probs = nullptr;
@@ -140,7 +140,7 @@ struct tt_ctx {
     int K = 0;
     tt_frame frames[TT_MAX_STREAMS];
     tt_state* states[TT_MAX_STREAMS];
-  } slots[2];
+  } slots[TT_MAX_IN_FLIGHT];
   int q_head = 0, q_count = 0;      // oldest in-flight slot, number in flight
   int bound = 0;                    // slot whose resources the view members hold
   int last_done = -1;               // slot of the last completed submit (debug taps)
@@ -162,12 +162,12 @@ struct tt_ctx {
   // Every slot owns a few device tables, each remembering the set of frame pointers it holds: a caller whose
   // frames arrive in a fixed set of buffers (a capture ring; the slot's own staging buffer for host frames) finds
   // its pointers already on the device and no copy is enqueued.
-  static constexpr int FRAME_TABS = 4;
-  const uint8_t** frame_tab_dev[2] = {nullptr, nullptr};   // device, [FRAME_TABS][TT_MAX_STREAMS] pointers per slot
-  const uint8_t** frame_tab_host[2] = {nullptr, nullptr};  // pinned staging of one table
-  const uint8_t* frame_tab_last[2][FRAME_TABS][TT_MAX_STREAMS] = {};   // what each device table holds
-  bool frame_tab_valid[2][FRAME_TABS] = {};
-  uint64_t frame_tab_used[2][FRAME_TABS] = {};             // tick at which the table was last used (the oldest is replaced)
+  static constexpr int FRAME_TABS = 8;
+  const uint8_t** frame_tab_dev[TT_MAX_IN_FLIGHT] = {};   // device, [FRAME_TABS][TT_MAX_STREAMS] pointers per slot
+  const uint8_t** frame_tab_host[TT_MAX_IN_FLIGHT] = {};  // pinned staging of one table
+  const uint8_t* frame_tab_last[TT_MAX_IN_FLIGHT][FRAME_TABS][TT_MAX_STREAMS] = {};   // what each device table holds
+  bool frame_tab_valid[TT_MAX_IN_FLIGHT][FRAME_TABS] = {};
+  uint64_t frame_tab_used[TT_MAX_IN_FLIGHT][FRAME_TABS] = {};             // tick at which the table was last used (the oldest is replaced)
   const uint8_t* const* cur_tab = nullptr;                  // table the tick being enqueued reads
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_copy = nullptr;
@@ -503,8 +503,8 @@ tt_status build(tt_ctx* ctx, const tt_weights* w) {
     if ((st = dev_alloc(ctx, &scr, post_scratch_bytes(S, ctx->Hm, ctx->Wm, ctx->Ch, ctx->T))) != TT_OK) return st;
     ctx->post_scratch = scr;
   }
-  // per-slot resources: two submits may be in flight
-  for (int i = 0; i < 2; ++i) {
+  // per-slot resources
+  for (int i = 0; i < TT_MAX_IN_FLIGHT; ++i) {
     tt_ctx::Slot& sl = ctx->slots[i];
     if ((st = dev_alloc(ctx, &sl.frames_stage, (size_t)S * ctx->frame_bytes + 16)) != TT_OK) return st;
     if ((st = dev_alloc(ctx, &sl.logits, (size_t)S * ctx->T * plane)) != TT_OK) return st;
@@ -673,7 +673,7 @@ void release(tt_ctx* ctx) {
   if (ctx->stream) cudaStreamSynchronize(ctx->stream);
   for (void* p : ctx->allocs) cudaFree(p);
   if (ctx->copy_stream) cudaStreamSynchronize(ctx->copy_stream);
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < TT_MAX_IN_FLIGHT; ++i) {
     tt_ctx::Slot& sl = ctx->slots[i];
     if (sl.results_host) cudaFreeHost(sl.results_host);
     if (sl.status_host) cudaFreeHost(sl.status_host);
@@ -685,7 +685,7 @@ void release(tt_ctx* ctx) {
   }
   for (auto& g : ctx->graphs)
     if (g.exec) cudaGraphExecDestroy(g.exec);
-  for (int i = 0; i < 2; ++i)
+  for (int i = 0; i < TT_MAX_IN_FLIGHT; ++i)
     if (ctx->frame_tab_host[i]) cudaFreeHost(ctx->frame_tab_host[i]);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   if (ctx->own_stream && ctx->stream) cudaStreamDestroy(ctx->stream);
@@ -1006,7 +1006,8 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
   if (!frames || !states || K < 1) return fail(ctx, TT_ERR_INVALID_ARG, "null frames/states or K < 1");
   if (K > ctx->cfg.max_streams)
     return fail(ctx, TT_ERR_ADMISSION, "K = %d streams exceed the %d this context was sized for", K, ctx->cfg.max_streams);
-  if (ctx->q_count >= 2) return fail(ctx, TT_ERR_NOT_READY, "two submits are already in flight; call tt_sync first");
+  if (ctx->q_count >= TT_MAX_IN_FLIGHT)
+    return fail(ctx, TT_ERR_NOT_READY, "%d submits are already in flight; call tt_sync first", TT_MAX_IN_FLIGHT);
   for (int n = 0; n < K; ++n) {
     if (!owns_state(ctx, states[n])) return fail(ctx, TT_ERR_INVALID_ARG, "states[%d] is null or belongs to another context", n);
     if (!frames[n].data) return fail(ctx, TT_ERR_INVALID_ARG, "frames[%d].data is null", n);
@@ -1014,7 +1015,7 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
       if (states[m] == states[n]) return fail(ctx, TT_ERR_INVALID_ARG, "states[%d] and states[%d] are the same state", m, n);
   }
   TT_CUDA(ctx, cudaSetDevice(ctx->dev));
-  const int slot = (ctx->q_head + ctx->q_count) & 1;   // the slot that is not in flight (or the only free one)
+  const int slot = (ctx->q_head + ctx->q_count) % TT_MAX_IN_FLIGHT;   // the oldest slot that is not in flight
   bind_slot(ctx, slot);
   cudaStream_t s = ctx->stream;
   TT_CUDA(ctx, cudaEventRecord(ctx->ev_start, s));
@@ -1083,7 +1084,7 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
       if (same) { tg = &g; break; }
     }
     if (!tg) {
-      if (ctx->graphs.size() >= 128) {            // bounded cache: drop everything and start over
+      if (ctx->graphs.size() >= 256) {            // bounded cache: drop everything and start over
         for (auto& g : ctx->graphs)
           if (g.exec) cudaGraphExecDestroy(g.exec);
         ctx->graphs.clear();
@@ -1172,7 +1173,7 @@ tt_status tt_sync(tt_ctx* ctx, tt_result* results) {
       std::this_thread::yield();
     }
   }
-  ctx->q_head ^= 1;
+  ctx->q_head = (ctx->q_head + 1) % TT_MAX_IN_FLIGHT;
   ctx->q_count -= 1;
   ctx->last_done = slot;
   float ms = 0.f;

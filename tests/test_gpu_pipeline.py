@@ -571,9 +571,10 @@ def test_dependent_launches_change_no_bit(cuda_device):
         assert np.array_equal(h1, h2) and np.array_equal(c1, c2)
 
 
-def test_two_submits_in_flight_match_serial_execution(cuda_device):
-    """Software-pipelined use (submit t+1 before sync t, pinned host frames over the copy stream) must give
-    bit for bit what one-at-a-time execution gives, with results returned oldest first."""
+@pytest.mark.parametrize("depth", [2, 3])
+def test_submits_in_flight_match_serial_execution(cuda_device, depth):
+    """Software-pipelined use (`depth` submits in flight: submit t+depth-1 before sync t, pinned host frames over the
+    copy stream) must give bit for bit what one-at-a-time execution gives, with results returned oldest first."""
     wl = tt_synth.workload("cfg1-gain").with_(name="pipe", src_w=214, src_h=120, net_w=160, net_h=120, overlay=True)
     K, n = 2, 6
     frames = [[torch.from_numpy(f).pin_memory() for f in fs] for fs in _frames(wl, K, n)]
@@ -591,11 +592,13 @@ def test_two_submits_in_flight_match_serial_execution(cuda_device):
 
     ctx, states, _ = _make(wl, K, overlay=True)
     piped = []
-    ctx.submit_frames([frames[k][0] for k in range(K)], states, frame_index=0)
-    for t in range(1, n):
+    for t in range(depth - 1):
         ctx.submit_frames([frames[k][t] for k in range(K)], states, frame_index=t)
-        piped.append(collect(ctx, ctx.sync()))          # results of tick t-1 while tick t is in flight
-    piped.append(collect(ctx, ctx.sync()))
+    for t in range(depth - 1, n):
+        ctx.submit_frames([frames[k][t] for k in range(K)], states, frame_index=t)
+        piped.append(collect(ctx, ctx.sync()))          # results of tick t-depth+1 while the later ones are in flight
+    while len(piped) < n:
+        piped.append(collect(ctx, ctx.sync()))
     h_piped = [ctx.state_export(s) for s in states]
     ctx.destroy()
     for t in range(n):
@@ -627,14 +630,17 @@ def test_boundary_error_paths(cuda_device):
     with pytest.raises(binding.TTError) as e:
         ctx.submit_frames([], [])
     assert e.value.status == 1
+    assert binding.TT_MAX_IN_FLIGHT == 3
     ctx.submit_frames([f], [st])
-    ctx.submit_frames([f], [st2])                               # a second submit may be in flight
+    ctx.submit_frames([f], [st2])                               # a second and a third submit may be in flight
+    ctx.submit_frames([f], [st])
     with pytest.raises(binding.TTError) as e:
         ctx.submit_frames([f], [st])
-    assert e.value.status == 6                                  # but not a third
+    assert e.value.status == 6                                  # but not a fourth
     with pytest.raises(binding.TTError) as e:
         ctx.state_reset(st)
     assert e.value.status == 6
+    assert len(ctx.sync()) == 1
     assert len(ctx.sync()) == 1
     with pytest.raises(binding.TTError) as e:
         ctx.state_export(st)

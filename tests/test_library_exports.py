@@ -97,3 +97,10 @@ def test_option_indices_in_the_binding_match_the_header():
     for name in dir(binding):
         if name.startswith("TT_OPT_"):
             assert name in declared, f"{name} is not in tt.h"
+
+
+def test_limits_in_the_binding_match_the_header():
+    text = open(os.path.join(ROOT, "include", "tt.h")).read()
+    for name in ("TT_MAX_STREAMS", "TT_MAX_TOOLS", "TT_MAX_ENC", "TT_MAX_IN_FLIGHT"):
+        (val,) = re.findall(r"#define\s+%s\s+(\d+)" % name, text)
+        assert getattr(binding, name) == int(val), name
