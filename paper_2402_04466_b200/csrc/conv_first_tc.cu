@@ -36,9 +36,12 @@ using namespace tc;
 constexpr int F_STAGES = 3;
 constexpr int F_A_BYTES = 128 * 64;                 // 128 rows x 32 bf16
 constexpr int F_THREADS = 288;                      // warps 0-3 gather, 4 MMA, 5-8 epilogue
-constexpr int F_THREADS_FUSED = F_THREADS + 128;    // warps 9-12 stage frame rows and sample them into the patch buffers
+constexpr int F_SAMPLER_WARPS = 8;                  // FUSED: warps 9.. stage frame rows and sample them into the patch buffers
+constexpr int F_SAMPLERS = 32 * F_SAMPLER_WARPS;
+constexpr int F_THREADS_FUSED = F_THREADS + F_SAMPLERS;
 constexpr int F_SRC_STAGES = 3;
-constexpr int F_SRC_PASSES = 4;                     // a staging pass moves 8 rows of up to 16 vectors: at most 32 rows of 256 bytes
+constexpr int F_SRC_ROWS = 32;                      // staged rows per tile at most, of up to 16 vectors (256 bytes) each
+constexpr int F_SRC_PASSES = F_SRC_ROWS / (F_SAMPLERS / 16);   // a staging pass moves one vector per sampler thread
 constexpr int F_SRC_BUDGET = 48 * 1024;             // shared memory the staged frame rows may take
 constexpr int F_MAX_TILES = 128;                    // tile columns and tile rows the fused form keeps source ranges for
 constexpr int F_TMEM_COLS = 128;                    // two accumulator buffers of up to 64 columns
@@ -84,10 +87,12 @@ conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
   uint8_t* s_b = s_a + F_STAGES * F_A_BYTES;                  // weights in operand layout
   uint8_t* s_patch = s_b + COUT * 64;                         // [2] patches of [3][PH][BW] floats
   uint8_t* s_src = s_patch + 2 * PATCH_STRIDE;                // FUSED: [F_SRC_STAGES] x src_rows_cap rows of src_row_cap bytes
+  // FUSED: sample positions of every patch column of every tile column {3 * left source column or -1 outside the image, fx}
+  // and of every patch row of every tile row {upper source row or -1, lower source row, fy, -}
+  int2* s_xtab = reinterpret_cast<int2*>(s_src + F_SRC_STAGES * p.src_rows_cap * p.src_row_cap);
+  int4* s_ytab = reinterpret_cast<int4*>(s_xtab + ((p.tiles_x * PW + 1) & ~1));
   __shared__ __align__(8) uint64_t s_bar[2 * F_STAGES + 8];
   __shared__ const uint8_t* s_frame[TT_MAX_STREAMS];          // the batch's frame pointers
-  __shared__ int s_yoff0[2][PH], s_yoff1[2][PH];              // per patch row: byte offsets of its two source rows' first staged column, -1 outside
-  __shared__ float s_fy[2][PH];
   __shared__ int s_gx[F_MAX_TILES][2], s_gy[F_MAX_TILES][2];  // first and last source column / row under every tile column / row
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
@@ -110,7 +115,7 @@ conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(t_full + a), 1);
       mbar_init(smem_u32(t_empty + a), 4);
-      mbar_init(smem_u32(p_full + a), FUSED ? 128 : 1);
+      mbar_init(smem_u32(p_full + a), FUSED ? F_SAMPLERS : 1);
       mbar_init(smem_u32(p_empty + a), 128);
     }
     s_abort = 0;
@@ -132,6 +137,20 @@ conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
         const int first = max(t * 8 * STRIDE - 1, 0), last = min(t * 8 * STRIDE - 1 + PH - 1, p.H - 1);
         s_gy[t][0] = pre::axis_sample(first, p.src_h, p.H).i0;
         s_gy[t][1] = pre::axis_sample(last, p.src_h, p.H).i1;
+      }
+    }
+    const float inv_den_x = 1.0f / (float)(2 * p.W), inv_den_y = 1.0f / (float)(2 * p.H);
+    for (int i = threadIdx.x; i < p.tiles_x * PW + p.tiles_y * PH; i += F_THREADS_FUSED) {
+      if (i < p.tiles_x * PW) {
+        const int t = i / PW, x = t * 16 * STRIDE - 1 + (i - t * PW);
+        const bool in = x >= 0 && x < p.W;
+        const pre::AxisSample sx = pre::axis_sample_fast(in ? x : 0, p.src_w, p.W, inv_den_x);
+        s_xtab[i] = make_int2(in ? 3 * sx.i0 : -1, __float_as_int(sx.f));
+      } else {
+        const int k = i - p.tiles_x * PW, t = k / PH, y = t * 8 * STRIDE - 1 + (k - t * PH);
+        const bool in = y >= 0 && y < p.H;
+        const pre::AxisSample sy = pre::axis_sample_fast(in ? y : 0, p.src_h, p.H, inv_den_y);
+        s_ytab[k] = make_int4(in ? sy.i0 : -1, sy.i1, __float_as_int(sy.f), 0);
       }
     }
   }
@@ -242,26 +261,34 @@ conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
   } else if (FUSED && warp >= 9) {
     // ------------------------------------------------------- frame samplers (preprocessing)
     // Patch entry (c, r, j + 3) is pixel (y_base + r, x_base + j) of the resized image, zero outside it (the
-    // convolution's padding).  Thread (g, j) of the first RG * PW owns patch column j and the rows g, g + RG, ...:
-    // its horizontal sample position is worked out once per tile and stays in registers.  The next PH threads work
-    // out the vertical positions of the tile's rows into shared memory meanwhile (one integer division per thread).
+    // convolution's padding).  Thread (g, j) of the first RG * PW owns patch column j and the rows g, g + RG, ...;
+    // sample positions come from the tables made at the start of the kernel.
     //
-    // Staging: in pass k thread t moves 16-byte vector t % 16 of footprint row t / 16 + 8k.  The stage written
-    // while tile i is handled (for tile i + 2) was last read for tile i - 1, which every thread has left behind
-    // at tile i's barrier; the same barrier, one tile later, makes the stores visible before they are read.
-    constexpr int RG = (128 - PH) / PW;
+    // Staging: in pass k thread t moves 16-byte vector t % 16 of footprint row t / 16 + (F_SAMPLERS / 16) k.  The
+    // stage written while tile i is handled (for tile i + 2) was last read for tile i - 1, which every thread has
+    // left behind at tile i's barrier; the same barrier, one tile later, makes the stores visible before they are read.
+    constexpr int RG = (F_SAMPLERS / PW) < PH ? (F_SAMPLERS / PW) : PH;
     constexpr int ROWS = (PH + RG - 1) / RG;
+    constexpr int VROWS = F_SAMPLERS / 16;
     const int bt = threadIdx.x - F_THREADS;
     const int g = bt / PW, j = bt - g * PW;
+    const bool active = g < RG;
     const int stage_bytes = p.src_rows_cap * p.src_row_cap;
     const int vrow = bt >> 4, vcol = bt & 15;
-    const float inv_den_x = 1.0f / (float)(2 * p.W), inv_den_y = 1.0f / (float)(2 * p.H);
     uint4 vreg[F_SRC_PASSES];
     uint32_t vmask = 0;
     uint32_t st = 0;   // stage of the current tile's rows
 
-    auto stage_load = [&](int tile) {
-      const TileAt t = tile_at(tile, p.tiles_x, tiles_per_img, inv_tiles_x, inv_tiles_per_img);
+    // tile coordinates advance by the grid size without divisions: the step's own decomposition, then two carries
+    const TileAt step = tile_at((int)gridDim.x, p.tiles_x, tiles_per_img, inv_tiles_x, inv_tiles_per_img);
+    auto advance = [&](TileAt& c) {
+      c.tx += step.tx;
+      if (c.tx >= p.tiles_x) { c.tx -= p.tiles_x; ++c.ty; }
+      c.ty += step.ty;
+      if (c.ty >= p.tiles_y) { c.ty -= p.tiles_y; ++c.img; }
+      c.img += step.img;
+    };
+    auto stage_load = [&](const TileAt& t) {
       const int sx_lo = s_gx[t.tx][0], sx_hi = s_gx[t.tx][1], sy_lo = s_gy[t.ty][0], sy_hi = s_gy[t.ty][1];
       const int n_rows = min(sy_hi - sy_lo + 1, p.src_rows_cap);
       const int span = 3 * (sx_hi - sx_lo) + 2;            // a row's bytes run from its first byte to first + span
@@ -271,54 +298,44 @@ conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
       for (int k = 0; k < F_SRC_PASSES; ++k) {
         const uintptr_t a_vec = (g_first & ~(uintptr_t)15) + (uintptr_t)vcol * 16;
         // the vector starts at or before the row's last byte and inside the staged row
-        if (vrow + 8 * k < n_rows && a_vec <= g_first + span && vcol < (p.src_row_cap >> 4)) {
+        if (vrow + VROWS * k < n_rows && a_vec <= g_first + span && vcol < (p.src_row_cap >> 4)) {
           vreg[k] = __ldg(reinterpret_cast<const uint4*>(a_vec));
           vmask |= 1u << k;
         }
-        g_first += (size_t)8 * p.src_pitch;
+        g_first += (size_t)VROWS * p.src_pitch;
       }
     };
     auto stage_store = [&](int st) {
       uint8_t* dst = s_src + st * stage_bytes + vrow * p.src_row_cap + vcol * 16;
 #pragma unroll
       for (int k = 0; k < F_SRC_PASSES; ++k)
-        if (vmask & (1u << k)) *reinterpret_cast<uint4*>(dst + 8 * k * p.src_row_cap) = vreg[k];
+        if (vmask & (1u << k)) *reinterpret_cast<uint4*>(dst + VROWS * k * p.src_row_cap) = vreg[k];
     };
 
+    TileAt cur = tile_at((int)blockIdx.x, p.tiles_x, tiles_per_img, inv_tiles_x, inv_tiles_per_img);
+    TileAt ahd = cur;
     // the first two tiles' rows
-    if (blockIdx.x < total_tiles) { stage_load(blockIdx.x); stage_store(0); }
-    if (blockIdx.x + gridDim.x < total_tiles) { stage_load(blockIdx.x + gridDim.x); stage_store(1); }
+    if (blockIdx.x < total_tiles) { stage_load(ahd); stage_store(0); }
+    advance(ahd);
+    if (blockIdx.x + gridDim.x < total_tiles) { stage_load(ahd); stage_store(1); }
+    advance(ahd);
     uint32_t it = 0;
     bool fail = false;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
       const int b = (int)(it & 1u);
-      const TileAt t = tile_at(tile, p.tiles_x, tiles_per_img, inv_tiles_x, inv_tiles_per_img);
-      const int x_base = t.tx * 16 * STRIDE - 1, y_base = t.ty * 8 * STRIDE - 1;
-      const int sx_lo = s_gx[t.tx][0], sy_lo = s_gy[t.ty][0];
       const bool ahead = tile + 2 * (int)gridDim.x < total_tiles;
-      if (ahead) stage_load(tile + 2 * gridDim.x);
-      int xo = -1;
-      float fx = 0.f;
-      if (g < RG) {
-        const int x = x_base + j;
-        if (x >= 0 && x < p.W) {
-          const pre::AxisSample sx = pre::axis_sample_fast(x, p.src_w, p.W, inv_den_x);
-          xo = 3 * (sx.i0 - sx_lo);
-          fx = sx.f;
-        }
-      } else if (bt < RG * PW + PH) {
-        const int r = bt - RG * PW, y = y_base + r;
-        const bool in = y >= 0 && y < p.H;
-        const pre::AxisSample sy = pre::axis_sample_fast(in ? y : 0, p.src_h, p.H, inv_den_y);
-        const uint32_t src_lo = (uint32_t)(uintptr_t)s_frame[t.img];   // only the low bits matter for 16-byte alignment
-        // byte position of source column sx_lo inside the two staged rows
-        s_yoff0[b][r] = in ? (sy.i0 - sy_lo) * p.src_row_cap + (int)((src_lo + (uint32_t)(sy.i0 * p.src_pitch + 3 * sx_lo)) & 15u) : -1;
-        s_yoff1[b][r] = in ? (sy.i1 - sy_lo) * p.src_row_cap + (int)((src_lo + (uint32_t)(sy.i1 * p.src_pitch + 3 * sx_lo)) & 15u) : -1;
-        s_fy[b][r] = sy.f;
-      }
+      if (ahead) stage_load(ahd);
+      const int sx_lo = s_gx[cur.tx][0], sy_lo = s_gy[cur.ty][0];
+      const int2 xe = active ? s_xtab[cur.tx * PW + j] : make_int2(-1, 0);
+      const int xo = xe.x >= 0 ? xe.x - 3 * sx_lo : -1;   // byte offset of the left tap from the first staged column
+      const float fx = __int_as_float(xe.y);
+      // low bits of the address of the first staged column in source row 0: (that + row * pitch) & 15 is the byte
+      // position of the column inside the staged row
+      const uint32_t base_lo = (uint32_t)(uintptr_t)s_frame[cur.img] + (uint32_t)(3 * sx_lo);
+      const int4* ytab = s_ytab + cur.ty * PH;
       if (!mbar_wait(smem_u32(p_empty + b), ((it >> 1) & 1u) ^ 1u, abort_flag, p.status, 0xA00 + b, wait_limit)) fail = true;
-      if (named_barrier_or(4, 128, fail)) break;
-      if (g < RG) {
+      if (named_barrier_or(4, F_SAMPLERS, fail)) break;
+      if (active) {
         const uint32_t* words = reinterpret_cast<const uint32_t*>(s_src + st * stage_bytes);
         float* d = reinterpret_cast<float*>(s_patch + b * PATCH_STRIDE) + j + 3;
 #pragma unroll
@@ -326,17 +343,19 @@ conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
           // rows behind the patch's last are computed like the last one and not stored; samples outside the image
           // are computed from the first staged bytes and replaced by zero: no branch but the one on fy
           const int r = g + k * RG, rc = min(r, PH - 1);
-          const int y0 = s_yoff0[b][rc];
-          const float fy = s_fy[b][rc];
-          const bool in = xo >= 0 && y0 >= 0;
+          const int4 ye = ytab[rc];
+          const float fy = __int_as_float(ye.z);
+          const bool in = xo >= 0 && ye.x >= 0;
+          const int off0 = (ye.x - sy_lo) * p.src_row_cap + (int)((base_lo + (uint32_t)(ye.x * p.src_pitch)) & 15u) + xo;
           float o0, o1, o2;
           uint32_t lo0, hi0;
-          fetch_pair(words, in ? y0 + xo : 0, lo0, hi0);
+          fetch_pair(words, in ? off0 : 0, lo0, hi0);
           if (fy == 0.0f) {
             pre::sample_row(lo0, hi0, fx, p.scale, p.shift, o0, o1, o2);
           } else {
+            const int off1 = (ye.y - sy_lo) * p.src_row_cap + (int)((base_lo + (uint32_t)(ye.y * p.src_pitch)) & 15u) + xo;
             uint32_t lo1, hi1;
-            fetch_pair(words, in ? s_yoff1[b][rc] + xo : 0, lo1, hi1);
+            fetch_pair(words, in ? off1 : 0, lo1, hi1);
             pre::sample_rows(lo0, hi0, lo1, hi1, fx, fy, p.scale, p.shift, o0, o1, o2);
           }
           if (r < PH) {
@@ -349,6 +368,8 @@ conv_first_tc_kernel(const __grid_constant__ ConvFirstTcParams p) {
       mbar_arrive(smem_u32(p_full + b));
       if (ahead) stage_store((int)(st == 0 ? 2 : st - 1));   // (it + 2) mod 3
       st = st == 2 ? 0 : st + 1;
+      advance(cur);
+      advance(ahd);
     }
   } else {
     // --------------------------------------------------------------------------- epilogue
@@ -418,7 +439,8 @@ template <int COUT, int STRIDE, bool FUSED>
 cudaError_t launch_t(const ConvFirstTcParams& p, int sm_count, cudaStream_t s) {
   constexpr int PH = 7 * STRIDE + 3;
   constexpr int SMEM = 1024 + 128 * COUT * 2 + F_STAGES * F_A_BYTES + COUT * 64 + 2 * ((3 * PH * box_w(STRIDE) * 4 + 127) & ~127);
-  const int smem = SMEM + (FUSED ? F_SRC_STAGES * p.src_rows_cap * p.src_row_cap : 0);
+  constexpr int PW = 15 * STRIDE + 3;
+  const int smem = SMEM + (FUSED ? F_SRC_STAGES * p.src_rows_cap * p.src_row_cap + 8 * ((p.tiles_x * PW + 1) & ~1) + 16 * p.tiles_y * PH : 0);
   const int total = p.K * p.tiles_x * p.tiles_y;
   const int slots = (FUSED ? 2 : 3) * sm_count;
   const int grid = total < slots ? total : slots;
@@ -454,10 +476,12 @@ bool conv_first_tc_staging(int stride, int src_w, int src_h, int net_w, int net_
   const long cap = ((3 * cols + 48 + 15) / 16) * 16;
   *rows_cap = (int)rows;
   *row_cap = (int)cap;
-  if (rows > 8 * F_SRC_PASSES || cap > 256) return false;   // what the staging passes of the kernel cover
+  if (rows > F_SRC_ROWS || cap > 256) return false;   // what the staging passes of the kernel cover
   // the sample positions are worked out with pre::div_by: numerators below 2^27
   if ((2L * net_w + 1) * src_w >= (1L << 27) || (2L * net_h + 1) * src_h >= (1L << 27)) return false;
-  return F_SRC_STAGES * rows * cap <= F_SRC_BUDGET;
+  // staged rows plus the tables of sample positions
+  const long tables = 8 * (((wo + 15) / 16 * pw + 1) & ~1L) + 16 * ((ho + 7) / 8) * ph;
+  return F_SRC_STAGES * rows * cap + tables <= F_SRC_BUDGET;
 }
 
 // [cout][27] bf16 bit patterns (row-major, k = c*9 + ky*3 + kx) -> operand layout, cout*32 values
