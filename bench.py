@@ -604,6 +604,9 @@ class Rig:
         from paper_2402_04466_b200 import binding
         for i in range(math.lcm(binding.TT_MAX_IN_FLIGHT, self.R, 2) + 1):
             self.tick(i, self.dev_ring)
+        if self.host_ring is not None:      # host frames pass through the slot's staging buffer: slots x halves
+            for i in range(math.lcm(binding.TT_MAX_IN_FLIGHT, 2) + 1):
+                self.tick(i, self.host_ring)
 
     def flush_l2(self, i):
         import torch
@@ -878,8 +881,8 @@ def run_ours(args):
                 "d2h_bytes_per_step": K * C.sizeof(binding.tt_result) + 4,
                 "value_with_l2_flush": n_frames / e2e_flush_s,
                 "serial_value": n_frames / e2e_serial_s,
-                "timing": "host clock, pinned host frames, host->device copies and the device->host result read inside. value: two "
-                          "submits in flight (tick i+1 submitted before tick i is synced), no cache flush (each step's input comes "
+                "timing": "host clock, pinned host frames, host->device copies and the device->host result read inside. value: three "
+                          "submits in flight (tick i+2 submitted before tick i is synced), no cache flush (each step's input comes "
                           "from host memory); value_with_l2_flush: the same with a 256 MiB flush write in stream order between ticks, "
                           "its time included; serial_value: submit -> sync one tick at a time, flush outside the timed part"},
         "gpu_launches": launches1 - launches0,
