@@ -87,17 +87,25 @@ __device__ __forceinline__ float fast_sigmoid(float z) { return fmaf(0.5f, fast_
 
 
 // ------------------------------------------------------------------------------------ kernel
-template <int BLOCK_N, int SLAB_C, int EPI, bool PAIR, int CTAS = 1, bool HALO = false>
+// WRES (weights resident): a layer whose whole packed weight matrix is at most WRES_BYTES fetches it once per
+// block, before it waits for the previous kernel, and the ring then holds activation boxes only: one copy per
+// iteration instead of two, and eight stages.
+constexpr int WRES_BYTES = 40 * 1024;
+constexpr int WRES_STAGES = 8;
+
+template <int BLOCK_N, int SLAB_C, int EPI, bool PAIR, int CTAS = 1, bool HALO = false, bool WRES = false>
 __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_constant__ ConvTcParams p) {
   using Cfg = TcCfg<BLOCK_N, SLAB_C, PAIR, CTAS>;
+  static_assert(!WRES || (!HALO && !PAIR && WRES_STAGES * Cfg::A_BYTES + WRES_BYTES + Cfg::BAR_BYTES + Cfg::TAB_BYTES + 1024 <= 112 * 1024),
+                "resident weights: single-CTA tap-box form that still fits twice on a multiprocessor");
   static_assert(!HALO || (SLAB_C == 64 && !PAIR && CTAS == 1), "halo mode: 64-channel slabs, one block per multiprocessor");
   constexpr int PW = HALO ? 8 : PATCH_W;           // output patch: 8 x 16 pixels in halo mode, 16 x 8 otherwise
   constexpr int PH = HALO ? 16 : PATCH_H;
   static_assert(CTAS == 1 || (CTAS == 2 && !PAIR && Cfg::TMEM_COLS <= 256 && Cfg::SMEM_BYTES <= 112 * 1024),
                 "two blocks per multiprocessor must fit its shared and tensor memory");
   // ring depth: stages of (A + B); in halo mode the weight ring, with the activation ring of its own behind it
-  constexpr int STAGES = HALO ? Cfg::HALO_B_STAGES : Cfg::STAGES;
-  constexpr int RING_STRIDE = HALO ? Cfg::B_BYTES : Cfg::STAGE_BYTES;
+  constexpr int STAGES = HALO ? Cfg::HALO_B_STAGES : WRES ? WRES_STAGES : Cfg::STAGES;
+  constexpr int RING_STRIDE = HALO ? Cfg::B_BYTES : WRES ? Cfg::A_BYTES : Cfg::STAGE_BYTES;
   constexpr int A_STAGES = Cfg::HALO_A_STAGES;
   constexpr uint32_t LAYOUT = SLAB_C == 64 ? 2u : 4u;
   constexpr uint32_t SBO = 8u * SLAB_C * 2u;
@@ -105,8 +113,8 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* smem_a = smem + STAGES * RING_STRIDE;               // halo mode: activation ring behind the weight ring
-  uint8_t* bar_mem = smem_a + (HALO ? A_STAGES * Cfg::HALO_A_BYTES : 0);
+  uint8_t* smem_a = smem + STAGES * RING_STRIDE;               // halo mode: activation ring behind the weight ring; WRES: the weights
+  uint8_t* bar_mem = smem_a + (HALO ? A_STAGES * Cfg::HALO_A_BYTES : WRES ? WRES_BYTES : 0);
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(bar_mem);   // [STAGES]
   uint64_t* empty_bar = full_bar + STAGES;                     // [STAGES]
   uint64_t* tfull_bar = empty_bar + STAGES;                    // [2]
@@ -177,6 +185,12 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&p.map_b) : "memory");
+    if (WRES) {
+      // all weight slabs, in iteration order, behind the ring; they land on the first "patch landed" barrier
+      const uint32_t wb = smem_u32(afull_bar);
+      mbar_arrive_expect_tx(wb, (uint32_t)(k_iters * Cfg::B_BYTES));
+      for (int it = 0; it < k_iters; ++it) tma_load_2d(smem_u32(smem_a + it * Cfg::B_BYTES), &p.map_b, wb, it * SLAB_C, 0);
+    }
   }
   if (warp == MMA_WARP) {
     __syncwarp();   // the table loop above may have left the warp's lanes apart; the allocation is warp-collective
@@ -262,7 +276,7 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
         const int4 e = s_tab[it];
         ok = mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag, p.status, 0x100 + (int)stage, wait_limit);
         if (!ok) break;
-        uint8_t* st = smem + stage * Cfg::STAGE_BYTES;
+        uint8_t* st = smem + stage * RING_STRIDE;
         if (PAIR) {
           const uint32_t fb = full0c + 8u * stage;
           mbar_arrive_expect_tx_cluster(fb, Cfg::STAGE_BYTES);
@@ -270,9 +284,9 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
           tma_load_2d_pair(smem_u32(st + Cfg::A_BYTES), &p.map_b, fb, it * SLAB_C, nt * BLOCK_N + rank * Cfg::B_ROWS);
         } else {
           const uint32_t fb = smem_u32(full_bar + stage);
-          mbar_arrive_expect_tx(fb, Cfg::STAGE_BYTES);
+          mbar_arrive_expect_tx(fb, WRES ? Cfg::A_BYTES : Cfg::STAGE_BYTES);
           tma_load_4d(smem_u32(st), maps + e.x * (int)sizeof(TensorMap128), fb, e.y, x0 + e.z, y0 + e.w, e.x < 4 ? img_x : img_h);
-          tma_load_2d(smem_u32(st + Cfg::A_BYTES), &p.map_b, fb, it * SLAB_C, nt * BLOCK_N);
+          if (!WRES) tma_load_2d(smem_u32(st + Cfg::A_BYTES), &p.map_b, fb, it * SLAB_C, nt * BLOCK_N);
         }
         stage += (uint32_t)n_prod;
         if (stage >= (uint32_t)STAGES) { stage -= STAGES; phase ^= 1u; }
@@ -289,7 +303,9 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
     int acc = 0;
     bool ok = true;
     const uint64_t a_desc0 = make_smem_desc(smem_u32(smem), SBO, LAYOUT);
-    constexpr uint64_t STAGE_UNITS = Cfg::STAGE_BYTES >> 4, B_UNITS = Cfg::A_BYTES >> 4;
+    constexpr uint64_t STAGE_UNITS = RING_STRIDE >> 4, B_UNITS = Cfg::A_BYTES >> 4;
+    const uint64_t w_desc0 = make_smem_desc(smem_u32(smem_a), SBO, LAYOUT);   // WRES: first resident weight slab
+    if (WRES) ok = mbar_wait(smem_u32(afull_bar), 0u, abort_flag, p.status, 0xB00, wait_limit);
     const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
     uint64_t a_desc = a_desc0;
     for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
@@ -333,7 +349,7 @@ __global__ void __launch_bounds__(TC_THREADS, CTAS) conv_tc_kernel(const __grid_
         // the copies complete on the barrier through the async proxy, which the MMAs read through too
         ok = mbar_wait(full0 + 8u * stage, phase, abort_flag, p.status, 0x300 + (int)stage, wait_limit);
         if (!ok) break;
-        const uint64_t b_desc = a_desc + B_UNITS;
+        const uint64_t b_desc = WRES ? w_desc0 + (uint64_t)it * (uint64_t)(Cfg::B_BYTES >> 4) : a_desc + B_UNITS;
         // advance along K inside the swizzle atom: 16 bf16 = 32 bytes = 2 descriptor units
         if (PAIR) {
           umma_bf16_pair(d_tmem, a_desc, b_desc, IDESC, it != 0 ? 1u : 0u);
@@ -500,6 +516,20 @@ cudaError_t launch_cfg(const ConvTcParams& p, int sm_count, cudaStream_t s) {
   return launch_kernel(kern, grid, TC_THREADS, Cfg::SMEM_BYTES, s, p, p.pdl != 0);
 }
 
+// Weights resident: two blocks per multiprocessor, ring of activation boxes, the whole weight matrix behind it.
+template <int BLOCK_N, int SLAB_C>
+cudaError_t launch_wres(const ConvTcParams& p, int sm_count, cudaStream_t s) {
+  using Cfg = TcCfg<BLOCK_N, SLAB_C, false, 2>;
+  constexpr int SMEM = WRES_STAGES * Cfg::A_BYTES + WRES_BYTES + Cfg::BAR_BYTES + Cfg::TAB_BYTES + 1024;
+  auto kern = conv_tc_kernel<BLOCK_N, SLAB_C, TC_EPI_RELU_BF16, false, 2, false, true>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  if (e != cudaSuccess) return e;
+  const int total_tiles = p.K * p.tiles_x * p.tiles_y;
+  const int slots = 2 * sm_count;
+  const int grid = total_tiles < slots ? total_tiles : slots;
+  return launch_kernel(kern, grid, TC_THREADS, SMEM, s, p, p.pdl != 0);
+}
+
 // CTA pairs: clusters of two, one pair per unit of work, as many pairs as the device can hold at once.
 template <int BLOCK_N, int SLAB_C, int EPI>
 cudaError_t launch_pair(const ConvTcParams& p, int sm_count, cudaStream_t s) {
@@ -560,6 +590,11 @@ cudaError_t launch_shape(const ConvTcParams& p, int sm_count, cudaStream_t s) {
   if (p.pair) {
     if (p.slab_c == 64 && p.block_n == 256) return launch_pair<256, 64, EPI>(p, sm_count, s);
     return cudaErrorInvalidValue;
+  }
+  if (EPI == TC_EPI_RELU_BF16 && p.two_per_sm && p.wres) {
+    const int k_iters = 9 * (p.slabs[0] + (p.n_src > 1 ? p.slabs[1] : 0));
+    if (p.slab_c != 32 || p.block_n != 64 || p.n_tiles_n != 1 || k_iters * 64 * 32 * 2 > WRES_BYTES) return cudaErrorInvalidValue;
+    return launch_wres<64, 32>(p, sm_count, s);
   }
   if (EPI == TC_EPI_RELU_BF16 && p.two_per_sm && p.block_n <= 128) {
     if (p.slab_c == 64 && p.block_n == 128) return launch_cfg<128, 64, TC_EPI_RELU_BF16, 2>(p, sm_count, s);

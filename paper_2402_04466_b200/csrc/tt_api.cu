@@ -811,6 +811,8 @@ tt_status enqueue_tick(tt_ctx* ctx, int K, const FramePtrs& frames, tt_state* co
       tt_status st = fill_common(q, L, ctx->lay_h[l + 1], ctx->lay_w[l + 1], true);
       if (st != TT_OK) return st;
       q.n_src = 1; q.slabs[0] = L.cin0 / L.slab_c; q.slabs[1] = 0; q.img0 = ident; q.img1 = ident;
+      // a weight matrix of at most 40 KB (64 outputs, up to 32 inputs x 9 taps) stays in shared memory for the whole launch
+      q.wres = (q.two_per_sm && q.block_n == 64 && L.slab_c == 32 && q.n_tiles_n == 1 && 9 * q.slabs[0] * 64 * 32 * 2 <= 40 * 1024) ? 1 : 0;
       q.epilogue = TC_EPI_RELU_BF16; q.out = reinterpret_cast<__nv_bfloat16*>(ctx->enc_out[l]);
       TT_CUDA(ctx, launch_conv_tc(q, ctx->sm_count, s));
       if ((ms_ = mark_stage(ctx, TT_STAGE_ENC0 + l, 1)) != TT_OK) return ms_;

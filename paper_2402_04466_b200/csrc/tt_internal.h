@@ -139,6 +139,7 @@ struct ConvTcParams {
   int32_t block_n;          // 64, 128 or 256
   int32_t n_prod;           // producer warps that issue loads, 1..3
   int32_t two_per_sm;       // encoder layers with tiles up to 128 wide: two blocks per multiprocessor, half the ring each
+  int32_t wres;             // two_per_sm layer of 64 outputs and 32-channel slabs whose weights fit in 40 KB: fetched once per block
   int32_t halo;             // stride-1 layer of 64-channel slabs: one haloed patch per channel slab, 8 x 16 output patches
   int32_t pair;             // run as CTA pairs (cta_group::2): block_n 256, map_b's box then holds 128 rows
   int32_t pdl;              // launch as a programmatic dependent of the previous kernel in the stream
