@@ -593,6 +593,7 @@ class Rig:
                   for sid in stream_ids]
         self.host_ring = [[f.pin_memory() for f in fs] for fs in frames] if host_frames else None
         self.dev_ring = [[f.to(dev) for f in fs] for fs in frames]
+        self.n_submits = 0
         self.settle()
 
     def settle(self):
@@ -613,9 +614,16 @@ class Rig:
         with torch.cuda.stream(self.stream):
             self.flush.fill_(i & 0xFF)
 
-    def tick(self, i, ring, K=None):
+    def submit(self, i, ring, K=None):
+        """Submit one tick.  The ring entry follows the context's own count of submits, not the caller's step index:
+        submit slot, state ping-pong half and frame buffer set then stay in step, and a context only ever meets the
+        lcm(slots, R, 2) graph keys it ran through while it was set up."""
         K = K or self.K
-        self.ctx.submit_frames([ring[s][i % self.R] for s in range(K)], self.states[:K], frame_index=i)
+        self.ctx.submit_frames([ring[s][self.n_submits % self.R] for s in range(K)], self.states[:K], frame_index=i)
+        self.n_submits += 1
+
+    def tick(self, i, ring, K=None):
+        self.submit(i, ring, K)
         return self.ctx.sync()
 
     def timed_ticks(self, steps, warmup):
@@ -755,7 +763,7 @@ def run_ours(args):
         for i in range(args.steps):
             if with_flush:
                 rig.flush_l2(i)
-            ctx.submit_frames([host_ring[s][i % R] for s in range(K)], states, frame_index=i)
+            rig.submit(i, host_ring)
             if i >= depth - 1:
                 last = ctx.sync()
         for _ in range(min(depth - 1, args.steps)):

@@ -145,7 +145,8 @@ typedef struct {
   const uint8_t* masks_dev;    /* device, [n_tools][Hm][Wm] 0/1; valid until submit number TT_MAX_IN_FLIGHT after this one */
   const float* probs_dev;      /* device, [n_tools][Hm][Wm]; same lifetime */
   const uint8_t* overlay_dev;  /* device, [src_h][src_w][4] RGBA8, or NULL when overlay is off */
-  float gpu_ms;                /* device time of the whole batch this frame was part of */
+  float gpu_ms;                /* device time of the whole batch this frame was part of: from the first thing the tick
+                                  enqueued (the host->device copies, for host frames) to its last */
   int32_t reserved_;
 } tt_result;
 

@@ -1020,10 +1020,21 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
   const int slot = (ctx->q_head + ctx->q_count) % TT_MAX_IN_FLIGHT;   // the oldest slot that is not in flight
   bind_slot(ctx, slot);
   cudaStream_t s = ctx->stream;
-  TT_CUDA(ctx, cudaEventRecord(ctx->ev_start, s));
   for (int i = 0; i < TT_STAGE_COUNT; ++i) ctx->stage_ran[i] = false;
   ctx->stage_valid = false;
   ctx->tick_profiled = ctx->profiling;
+  // The tick's start event goes in front of the first thing the tick enqueues.  With host frames or stage events that
+  // is here; a tick of device-resident frames records it only when its launch is ready, so that the host work in
+  // between (table look-ups, a graph capture) does not sit inside the device interval that gpu_ms reports.
+  bool start_pending = true;
+  auto record_start = [&]() -> cudaError_t {
+    if (!start_pending) return cudaSuccess;
+    start_pending = false;
+    return cudaEventRecord(ctx->ev_start, s);
+  };
+  bool any_host = ctx->profiling;
+  for (int n = 0; n < K; ++n) any_host |= !frames[n].on_device;
+  if (any_host) TT_CUDA(ctx, record_start());
   if (ctx->profiling) TT_CUDA(ctx, cudaEventRecord(ctx->stage_ev[0], s));
   FramePtrs fp{};
   bool any_h2d = false;
@@ -1054,19 +1065,24 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
     if (same) tab = i;
     if (ctx->frame_tab_used[slot][i] < ctx->frame_tab_used[slot][oldest]) oldest = i;
   }
-  if (tab < 0) {
-    tab = oldest;
-    for (int n = 0; n < TT_MAX_STREAMS; ++n) ctx->frame_tab_last[slot][tab][n] = ctx->frame_tab_host[slot][n] = n < K ? fp.p[n] : nullptr;
-    ctx->frame_tab_valid[slot][tab] = false;   // stays so if the copy cannot be enqueued
-    TT_CUDA(ctx, cudaMemcpyAsync(ctx->frame_tab_dev[slot] + tab * TT_MAX_STREAMS, ctx->frame_tab_host[slot],
-                                 sizeof(void*) * TT_MAX_STREAMS, cudaMemcpyHostToDevice, s));
-    ctx->frame_tab_valid[slot][tab] = true;
-  }
+  const bool tab_miss = tab < 0;
+  if (tab_miss) tab = oldest;
   ctx->frame_tab_used[slot][tab] = ctx->n_ticks + 1;
   ctx->cur_tab = ctx->frame_tab_dev[slot] + tab * TT_MAX_STREAMS;
-  // everything that moves host data to the device (frames, pointer table) counts as the H2D stage
-  st = mark_stage(ctx, TT_STAGE_H2D, 0);
-  if (st != TT_OK) return st;
+  // refreshes the chosen table; called in front of the tick's launch (a graph capture, which enqueues nothing,
+  // comes before it, so that its host time stays outside the interval between the tick's events)
+  auto refresh_table = [&]() -> tt_status {
+    TT_CUDA(ctx, record_start());
+    if (tab_miss) {
+      for (int n = 0; n < TT_MAX_STREAMS; ++n) ctx->frame_tab_last[slot][tab][n] = ctx->frame_tab_host[slot][n] = n < K ? fp.p[n] : nullptr;
+      ctx->frame_tab_valid[slot][tab] = false;   // stays so if the copy cannot be enqueued
+      TT_CUDA(ctx, cudaMemcpyAsync(ctx->frame_tab_dev[slot] + tab * TT_MAX_STREAMS, ctx->frame_tab_host[slot],
+                                   sizeof(void*) * TT_MAX_STREAMS, cudaMemcpyHostToDevice, s));
+      ctx->frame_tab_valid[slot][tab] = true;
+    }
+    // everything that moves host data to the device (frames, pointer table) counts as the H2D stage
+    return mark_stage(ctx, TT_STAGE_H2D, 0);
+  };
 
   // The launch sequence of a tick is replayed from a CUDA graph.  Which kernel variants a tick launches depends
   // on the stream count and the frames' alignment alone, so the first tick of such a family runs as plain
@@ -1099,6 +1115,7 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
     }
   }
   if (tg && tg->exec) {
+    if ((st = refresh_table()) != TT_OK) return st;
     TT_CUDA(ctx, cudaGraphLaunch(tg->exec, s));
     ctx->n_launches += tg->launches;
     ctx->n_ticks += 1;
@@ -1125,15 +1142,18 @@ tt_status tt_submit_frames(tt_ctx* ctx, int32_t K, const tt_frame* frames, tt_st
       ctx->graphs_off = true;
       ctx->n_launches = launches_before;
       ctx->n_ticks -= (st == TT_OK) ? 1 : 0;
+      if ((st = refresh_table()) != TT_OK) return st;
       st = enqueue_tick(ctx, K, fp, states);
       if (st != TT_OK) return st;
       TT_CUDA(ctx, cudaMemcpyAsync(ctx->results_host, ctx->results_dev, sizeof(tt_result) * K, cudaMemcpyDeviceToHost, s));
       TT_CUDA(ctx, cudaMemcpyAsync(ctx->status_host, ctx->status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
     } else {
       tg->launches = ctx->n_launches - launches_before;
+      if ((st = refresh_table()) != TT_OK) return st;
       TT_CUDA(ctx, cudaGraphLaunch(tg->exec, s));
     }
   } else {
+    if ((st = refresh_table()) != TT_OK) return st;
     st = enqueue_tick(ctx, K, fp, states);
     if (st != TT_OK) return st;
     TT_CUDA(ctx, cudaMemcpyAsync(ctx->results_host, ctx->results_dev, sizeof(tt_result) * K, cudaMemcpyDeviceToHost, s));

@@ -14,10 +14,11 @@ pytestmark = pytest.mark.gpu
 
 
 def _make(wl, K=1, overlay=None, precision=None, timeout_ns=0, plain_launches=False, cta_pairs=False, halo=True,
-          fused_pre=False):
+          fused_pre=False, enc_two_per_sm=True):
     weights = tt_synth.make_weights(wl)
     cfg = binding.make_config(wl, max_streams=K, overlay=overlay, precision=precision, sync_timeout_ns=timeout_ns,
-                              plain_launches=plain_launches, cta_pairs=cta_pairs, halo=halo, fused_pre=fused_pre)
+                              plain_launches=plain_launches, cta_pairs=cta_pairs, halo=halo, fused_pre=fused_pre,
+                              enc_two_per_sm=enc_two_per_sm)
     ctx = binding.Context(cfg, weights)
     states = [ctx.state_create() for _ in range(K)]
     return ctx, states, weights
@@ -338,6 +339,33 @@ def test_bf16_preprocessing_inside_the_first_layer_changes_no_bit(cuda_device, s
             res = ctx.sync()
             out.append([(ctx.fetch_probs(r), ctx.fetch_masks(r), ctx.fetch_overlay(r), r["conf"].copy(), r["cx"].copy(),
                          ctx.debug_tensor(states[i], "pre"), ctx.debug_tensor(states[i], "enc0")) for i, r in enumerate(res)])
+        runs.append((out, [ctx.state_export(s) for s in states]))
+        ctx.destroy()
+    (a, ha), (b, hb) = runs
+    for ta, tb in zip(a, b):
+        for ra, rb in zip(ta, tb):
+            for va, vb in zip(ra, rb):
+                assert np.array_equal(va, vb)
+    for (h1, c1), (h2, c2) in zip(ha, hb):
+        assert np.array_equal(h1, h2) and np.array_equal(c1, c2)
+
+
+def test_bf16_encoder_launch_shapes_change_no_bit(cuda_device):
+    """The tensor-core encoder layers run two blocks per multiprocessor by default, the 32 -> 64 channel layer with its
+    weights resident in shared memory; with one block per multiprocessor (weights streamed with the activations) the
+    products are accumulated in the same order, so every output and the state must be the same bits."""
+    wl = tt_synth.workload("cfg1-gain").with_(name="shapes", src_w=330, src_h=250, net_w=264, net_h=200, overlay=True)
+    K, n = 3, 3
+    host = _frames(wl, K, n)
+    runs = []
+    for two in (True, False):
+        ctx, states, _ = _make(wl, K, overlay=True, enc_two_per_sm=two)
+        out = []
+        for t in range(n):
+            ctx.submit_frames([torch.from_numpy(host[k][t]).to(cuda_device) for k in range(K)], states, frame_index=t)
+            res = ctx.sync()
+            out.append([(ctx.fetch_probs(r), ctx.fetch_masks(r), ctx.fetch_overlay(r), r["conf"].copy(), r["cx"].copy(),
+                         ctx.debug_tensor(states[i], "enc1"), ctx.debug_tensor(states[i], "enc2")) for i, r in enumerate(res)])
         runs.append((out, [ctx.state_export(s) for s in states]))
         ctx.destroy()
     (a, ha), (b, hb) = runs
